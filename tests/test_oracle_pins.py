@@ -1,0 +1,494 @@
+"""Pins for the float64 oracle: closed forms, invariants, library cross-checks and
+brute force on tiny inputs.  None of these tests touches the CUDA path."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+
+LN2 = math.log(2.0)
+rng = np.random.default_rng(1234)
+
+
+def rand_dist(V, sparsity=0.0):
+    p = rng.random(V) ** 3
+    if sparsity:
+        p[rng.random(V) < sparsity] = 0.0
+        p[rng.integers(V)] += 0.1
+    return p / p.sum()
+
+
+def bf16_bits(x):
+    """float array -> bf16 bits (round to nearest even), as the generator would store it."""
+    u = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+    return u.astype(np.uint16)
+
+
+# ------------------------------------------------------------------ softmax / entropy
+
+def test_softmax_golden_and_shift(golden):
+    c = golden["entropy_of_softmax_log1234"]
+    p, lse = oracle.softmax(c["z"])
+    assert np.allclose(p, c["expect"]["p"], atol=1e-15)
+    assert abs(lse - c["expect"]["lse"]) < 1e-14
+    assert abs(oracle.entropy(p) - c["expect"]["H"]) < 1e-14
+    z = rng.normal(size=1000) * 5
+    p0, l0 = oracle.softmax(z)
+    p1, l1 = oracle.softmax(z + 37.5)
+    assert np.allclose(p0, p1, atol=1e-15) and abs(l1 - l0 - 37.5) < 1e-12
+    assert abs(p0.sum() - 1.0) < 1e-13
+
+
+def test_softmax_matches_scipy():
+    from scipy.special import logsumexp, softmax
+    z = rng.normal(size=5000) * 4
+    p, lse = oracle.softmax(z)
+    assert np.allclose(p, softmax(z), rtol=1e-13, atol=0)
+    assert abs(lse - logsumexp(z)) < 1e-12
+
+
+def test_softmax_minus_inf_and_nan():
+    p, lse = oracle.softmax([0.0, -np.inf, 1.0, -np.inf])
+    assert p[1] == 0.0 and p[3] == 0.0 and abs(p.sum() - 1) < 1e-15
+    p, lse = oracle.softmax([-np.inf] * 4)
+    assert np.isnan(lse) and np.isnan(p).all()
+    p, lse = oracle.softmax([0.0, np.nan, 1.0])
+    assert np.isnan(lse)
+
+
+@pytest.mark.parametrize("V", [4, 1000, 128256])
+def test_entropy_uniform_is_ln_v(V):
+    assert abs(oracle.entropy(np.full(V, 1.0 / V)) - math.log(V)) < 1e-10
+    p, _ = oracle.softmax(np.full(V, 3.25))
+    assert abs(oracle.entropy(p) - math.log(V)) < 1e-10
+
+
+def test_entropy_onehot_and_golden(golden):
+    e = np.zeros(17)
+    e[5] = 1.0
+    assert oracle.entropy(e) == 0.0
+    c = golden["entropy_dyadic"]
+    assert abs(oracle.entropy(c["p"]) - c["expect"]["H"]) < 1e-15
+
+
+def test_entropy_equals_lse_minus_mean_logit():
+    z = rng.normal(size=3000) * 3
+    p, lse = oracle.softmax(z)
+    assert abs(oracle.entropy(p) - (lse - float(np.dot(p, z)))) < 1e-11
+
+
+def test_entropy_matches_scipy():
+    from scipy.stats import entropy
+    p = rand_dist(4096, 0.3)
+    assert abs(oracle.entropy(p) - entropy(p)) < 1e-12
+
+
+# ------------------------------------------------------------------ CE / KL / JSD / distance
+
+def test_kl_is_ce_minus_h(golden):
+    c = golden["kl_ce_dyadic_vs_uniform"]
+    assert abs(oracle.cross_entropy(c["p"], c["q"]) - c["expect"]["CE"]) < 1e-15
+    assert abs(oracle.kl(c["p"], c["q"]) - c["expect"]["KL"]) < 1e-15
+    for _ in range(5):
+        p, q = rand_dist(500), rand_dist(500)
+        assert abs(oracle.kl(p, q) - (oracle.cross_entropy(p, q) - oracle.entropy(p))) < 1e-12
+    # asymmetric: a transposed operand would be caught here
+    p, q = np.array([0.9, 0.1]), np.array([0.5, 0.5])
+    assert abs(oracle.kl(p, q) - (0.9 * math.log(1.8) + 0.1 * math.log(0.2))) < 1e-15
+    assert abs(oracle.kl(q, p) - (0.5 * math.log(0.5 / 0.9) + 0.5 * math.log(5.0))) < 1e-15
+
+
+def test_jsd_golden(golden):
+    for name in ("jsd_half_vs_onehot", "jsd_dyadic_vs_uniform", "jsd_disjoint"):
+        c = golden[name]
+        J = oracle.jsd(c["p"], c["q"])
+        assert abs(J - c["expect"]["JSD"]) < 1e-15, name
+        if "d" in c["expect"]:
+            assert abs(oracle.js_distance(J) - c["expect"]["d"]) < 1e-15, name
+
+
+def test_jsd_zero_symmetric_bounded():
+    for V in (4, 64, 5000):
+        p, q = rand_dist(V, 0.2), rand_dist(V, 0.2)
+        assert oracle.jsd(p, p) == 0.0
+        assert oracle.js_distance(oracle.jsd(p, p)) == 0.0
+        assert abs(oracle.jsd(p, q) - oracle.jsd(q, p)) < 1e-15
+        assert 0.0 <= oracle.jsd(p, q) <= LN2
+    # disjoint supports: exactly ln 2, distance exactly 1
+    p = np.zeros(100)
+    q = np.zeros(100)
+    p[:50] = rand_dist(50)
+    q[50:] = rand_dist(50)
+    assert abs(oracle.jsd(p, q) - LN2) < 1e-15
+    assert oracle.js_distance(LN2) == 1.0
+    assert oracle.js_distance(LN2 + 1e-9) == 1.0 and oracle.js_distance(-1e-12) == 0.0
+
+
+def test_jsd_two_printed_forms_agree():
+    for V in (4, 333, 20000):
+        p, q = rand_dist(V, 0.1), rand_dist(V, 0.1)
+        assert abs(oracle.jsd(p, q) - oracle.jsd_entropy_form(p, q)) < 1e-12
+        m = 0.5 * (p + q)
+        assert abs(oracle.jsd(p, q) - 0.5 * (oracle.kl(p, m) + oracle.kl(q, m))) < 1e-13
+
+
+def test_js_distance_matches_scipy_base2():
+    from scipy.spatial.distance import jensenshannon
+    for V in (4, 1000):
+        p, q = rand_dist(V), rand_dist(V)
+        assert abs(oracle.js_distance(oracle.jsd(p, q)) - jensenshannon(p, q, base=2)) < 1e-12
+
+
+def test_js_distance_is_sqrt_and_metric():
+    assert abs(oracle.js_distance(0.3) - math.sqrt(0.3 / LN2)) < 1e-15
+    for V in (4, 16, 64):
+        for _ in range(50):
+            a, b, c = rand_dist(V, 0.2), rand_dist(V, 0.2), rand_dist(V, 0.2)
+            d = lambda x, y: oracle.js_distance(oracle.jsd(x, y))
+            assert d(a, c) <= d(a, b) + d(b, c) + 1e-12
+
+
+# ------------------------------------------------------------------ inverse CDF
+
+def brute_inv_cdf(p, u):
+    c = 0.0
+    for v, pv in enumerate(p):
+        c += pv
+        if c > u:
+            return v
+    return max(v for v, pv in enumerate(p) if pv > 0)
+
+
+def test_inv_cdf_bruteforce_v4():
+    p = np.array([0.1, 0.2, 0.3, 0.4])
+    for u, want in [(0.0, 0), (0.05, 0), (0.11, 1), (0.29, 1), (0.31, 2), (0.59, 2), (0.61, 3),
+                    (0.999, 3)]:
+        assert oracle.inv_cdf(p, u)[0] == want
+    for u in np.linspace(0, 0.99999, 997):
+        for pp in (p, np.array([0.0, 0.5, 0.0, 0.5]), np.array([0.25] * 4)):
+            assert oracle.inv_cdf(pp, u)[0] == brute_inv_cdf(pp, u)
+
+
+def test_inv_cdf_margin_zero_mass_and_fallback():
+    p = np.array([0.0, 0.5, 0.0, 0.5])
+    v, m = oracle.inv_cdf(p, 0.3)
+    assert v == 1 and abs(m - 0.2) < 1e-15
+    v, m = oracle.inv_cdf(p, 0.5)      # C_1 = 0.5 is not > 0.5; token 2 has no mass
+    assert v == 3 and abs(m - 0.0) < 1e-15
+    # rounding leaves total mass below u: fall back to the last token with mass
+    p = np.array([0.3, 0.3, 0.3999999, 0.0])
+    assert oracle.inv_cdf(p, 0.99999999)[0] == 2
+
+
+def test_inv_cdf_histogram():
+    p = rand_dist(16)
+    us = (np.arange(200000) + 0.5) / 200000
+    counts = np.bincount([oracle.inv_cdf(p, u)[0] for u in us[::10]], minlength=16)
+    assert np.abs(counts / counts.sum() - p).max() < 2e-4
+
+
+# ------------------------------------------------------------------ KDE and Bayes
+
+def test_kde_golden(golden):
+    c = golden["kde_three_point"]
+    L = c["list"]
+    assert abs(oracle.sample_std(L) - c["expect"]["std"]) < 1e-15
+    assert abs(oracle.kde_bandwidth(L, 0) - c["expect"]["h_silverman"]) < 1e-15
+    assert abs(oracle.kde_bandwidth(L, 1) - c["expect"]["h_scott"]) < 1e-15
+    assert abs(oracle.kde(L, 0.4) - c["expect"]["f_0.4"]) < 1e-14
+    assert abs(oracle.kde(L, 0.2) - c["expect"]["f_0.2"]) < 1e-14
+    assert abs(oracle.kde(L, 0.6) - c["expect"]["f_0.2"]) < 1e-14   # symmetric list
+
+
+def test_kde_integrates_to_one_and_matches_scipy():
+    from scipy.stats import gaussian_kde
+    L = rng.random(40) * 0.8 + 0.1
+    xs = np.linspace(-2, 3, 20001)
+    f = np.array([oracle.kde(L, x) for x in xs])
+    assert abs(np.trapezoid(f, xs) - 1.0) < 1e-6
+    for rule, name in ((0, "silverman"), (1, "scott")):
+        g = gaussian_kde(L, bw_method=name)
+        for x in (0.0, 0.13, 0.5, 0.77, 1.0):
+            assert abs(oracle.kde(L, x, rule) - g(x)[0]) < 1e-12 * max(1.0, g(x)[0])
+
+
+def test_accept_prob_properties():
+    L = rng.random(30)
+    for d in (0.1, 0.5, 0.9):
+        # identical densities: posterior equals the prior
+        assert abs(oracle.accept_prob(L, L, d) - 0.5) < 1e-14
+    LA, LR = rng.random(50) * 0.5, 0.4 + rng.random(20) * 0.6
+    for d in (0.05, 0.3, 0.45, 0.7, 0.95):
+        pa = oracle.accept_prob(LA, LR, d)
+        pr = oracle.accept_prob(LR, LA, d)         # roles swapped: P(R|d)
+        assert abs(pa + pr - 1.0) < 1e-13
+        fa, fr = oracle.kde(LA, d), oracle.kde(LR, d)
+        assert abs(pa - 50 * fa / (50 * fa + 20 * fr)) < 1e-14
+    assert oracle.accept_prob(LA, LR, 0.1) > 0.9 and oracle.accept_prob(LA, LR, 0.9) < 0.1
+
+
+def test_accept_prob_cold_start():
+    L = rng.random(10)
+    assert oracle.accept_prob([], [], 0.3) == 0.0
+    assert oracle.accept_prob(L, [], 0.3) == 0.0
+    assert oracle.accept_prob(L, [0.4], 0.3) == 0.0
+    assert oracle.accept_prob([0.2], L, 0.3) == 0.0
+    assert oracle.accept_prob(L, [0.4, 0.4], 0.3) == 0.0          # zero deviation
+    assert oracle.accept_prob(L, L, 0.3, min_samples=11) == 0.0
+    assert oracle.accept_prob(L, L, 0.3, min_samples=10) == 0.5
+
+
+# ------------------------------------------------------------------ draft step
+
+def test_draft_step_strict_stop_and_sample():
+    z = np.zeros(4, dtype=np.float32)
+    r = oracle.draft_step(z, 0.6, 0.0)
+    assert abs(r["H"] - math.log(4)) < 1e-15 and r["stop"] and r["token"] == 2
+    assert not oracle.draft_step(z, 0.6, r["H"])["stop"]              # H == T_G: strict >
+    assert oracle.draft_step(z, 0.6, np.nextafter(r["H"], 0))["stop"]
+    zb = bf16_bits(np.log([1, 2, 3, 4]))
+    r = oracle.draft_step(zb, 0.35, 10.0)
+    zw = oracle.widen(zb)
+    p, lse = oracle.softmax(zw)
+    assert abs(r["H"] - oracle.entropy(p)) < 1e-15 and abs(r["lse"] - lse) < 1e-15
+    assert r["token"] == brute_inv_cdf(p, 0.35) and not r["stop"]
+
+
+def test_widen_bf16_exact():
+    x = np.array([1.0, -2.5, 0.15625, -np.inf, 3.0e38], dtype=np.float32)
+    b = bf16_bits(x)
+    w = oracle.widen(b)
+    assert w[0] == 1.0 and w[1] == -2.5 and w[2] == 0.15625 and w[3] == -np.inf
+    assert abs(w[4] / 3.0e38 - 1) < 2 ** -8
+
+
+# ------------------------------------------------------------------ Algorithm 1, brute force
+
+def py_alg1_round(state, zd, zt, x, ut, ua, min_samples=2):
+    """Independent statement of Alg. 1's verify + update with numpy/scipy routines.
+
+    state: dict with python lists LE, LA, LR and float T_G.  Uses scipy's softmax,
+    Jensen-Shannon distance and gaussian_kde, none of which the oracle calls."""
+    from scipy.spatial.distance import jensenshannon
+    from scipy.special import softmax
+    from scipy.stats import gaussian_kde
+    K = len(x)
+    P = [softmax(np.asarray(r, dtype=np.float64)) for r in zt]
+    Q = [softmax(np.asarray(r, dtype=np.float64)) for r in zd]
+    y = [brute_inv_cdf(P[i], float(ut[i])) for i in range(K + 1)]
+    w = K
+    for i in range(K):
+        d = float(jensenshannon(P[i], Q[i], base=2))
+        LA, LR = state["LA"], state["LR"]
+        if len(LA) >= max(2, min_samples) and len(LR) >= max(2, min_samples) \
+                and np.std(LA) > 0 and np.std(LR) > 0:
+            fa = gaussian_kde(LA, bw_method="silverman")(d)[0]
+            fr = gaussian_kde(LR, bw_method="silverman")(d)[0]
+            na, nr = len(LA), len(LR)
+            den = fa * na + fr * nr
+            pa = fa * na / den if den > 0 else 0.0
+        else:
+            pa = 0.0
+        if x[i] != y[i] and float(ua[i]) >= pa:
+            q = Q[i]
+            state["LE"].append(float(-(q[q > 0] * np.log(q[q > 0])).sum()))
+            if 0 < d < 1:
+                LR.append(d)
+            w = i
+            break
+        if 0 < d < 1:
+            LA.append(d)
+    if state["LE"]:
+        state["T_G"] = float(np.mean(state["LE"]))
+    return w, y[w]
+
+
+def test_alg1_trajectory_against_independent_python():
+    V, K, rounds = 48, 6, 60
+    r = np.random.default_rng(7)
+    st = oracle.SequenceState(capacity=1024, min_samples=8)   # longer cold start: more rejections
+    py = dict(LE=[], LA=[], LR=[], T_G=0.0)
+    n_rej = 0
+    for t in range(rounds):
+        zd = (r.normal(size=(K, V)) * 2).astype(np.float32)
+        zt = (zd + r.normal(size=(K, V)) * r.choice([0.1, 0.5, 1.5], size=(K, 1))).astype(np.float32)
+        zt = np.concatenate([zt, r.normal(size=(1, V)).astype(np.float32)])
+        ut = r.random(K + 1).astype(np.float32)
+        ua = r.random(K).astype(np.float32)
+        # draft tokens: mostly agree with the target sample so that windows vary
+        x = np.array([brute_inv_cdf(oracle.softmax(zt[i].astype(np.float64))[0], float(ut[i]))
+                      if r.random() < 0.8 else int(r.integers(V)) for i in range(K)])
+        out = oracle.verify_round(st, zd, zt, x, ut, ua)
+        w, tok = py_alg1_round(py, zd, zt, x, ut, ua, min_samples=8)
+        assert out["accept_len"] == w and out["next_token"] == tok, t
+        LE, LA, LR = st.lists()
+        assert np.allclose(LE, py["LE"], atol=1e-12) and len(LE) == len(py["LE"])
+        assert np.allclose(LA, py["LA"], atol=1e-12) and len(LA) == len(py["LA"])
+        assert np.allclose(LR, py["LR"], atol=1e-12) and len(LR) == len(py["LR"])
+        assert abs(st.T_G.value - py["T_G"]) < 1e-12
+        n_rej += out["rejected"]
+    assert 5 < n_rej < rounds and st.nA.value > 20 and st.nR.value > 5   # both regimes exercised
+
+
+def test_tg_is_running_mean_and_zero_until_first_rejection():
+    V, K = 32, 3
+    r = np.random.default_rng(3)
+    st = oracle.SequenceState(capacity=256, min_samples=1000)   # stay in the token-match regime
+    Hs = []
+    for t in range(12):
+        zd = r.normal(size=(K, V)).astype(np.float32)
+        zt = r.normal(size=(K + 1, V)).astype(np.float32)
+        ut = r.random(K + 1).astype(np.float32)
+        y = [oracle.inv_cdf(oracle.softmax(zt[i].astype(np.float64))[0], ut[i])[0] for i in range(K)]
+        x = np.array(y)
+        if t >= 4:                       # from round 4 on, break the match at position t % K
+            x[t % K] = (y[t % K] + 1) % V
+        out = oracle.verify_round(st, zd, zt, x, ut, np.zeros(K, dtype=np.float32) + 0.5)
+        if t < 4:
+            assert out["accept_len"] == K and not out["rejected"] and st.T_G.value == 0.0
+            assert out["next_token"] == out["y"][K]
+        else:
+            i = t % K
+            assert out["accept_len"] == i and out["rejected"] and out["next_token"] == y[i]
+            Hs.append(out["H_d"][i])
+            assert abs(st.T_G.value - np.mean(Hs)) < 1e-13
+    assert st.nE.value == 8
+
+
+def test_boundary_distances_skip_kde_lists_but_entropy_is_recorded():
+    V = 8
+    st = oracle.SequenceState(capacity=64)
+    same = np.array([[0.0, 1.0, 2.0, 3.0, -1.0, 0.5, 0.25, 2.5]], dtype=np.float32)
+    zt = np.concatenate([same, same])
+    # identical rows: d == 0; force a mismatch -> rejected (cold start P=0)
+    y0 = oracle.inv_cdf(oracle.softmax(same[0].astype(np.float64))[0], 0.5)[0]
+    out = oracle.verify_round(st, same, zt, [(y0 + 1) % V], [0.5, 0.5], [0.9])
+    assert out["dist"][0] == 0.0 and out["rejected"] and out["accept_len"] == 0
+    assert (st.nE.value, st.nA.value, st.nR.value) == (1, 0, 0)
+    assert abs(st.T_G.value - out["H_d"][0]) < 1e-15
+    # identical rows, matching token: accepted, still not recorded
+    out = oracle.verify_round(st, same, zt, [y0], [0.5, 0.5], [0.9])
+    assert out["accept_len"] == 1 and (st.nE.value, st.nA.value, st.nR.value) == (1, 0, 0)
+    # disjoint supports: d == 1
+    ninf = -np.inf
+    zd = np.array([[0.0, 1.0, ninf, ninf, ninf, ninf, ninf, ninf]], dtype=np.float32)
+    zt2 = np.array([[ninf, ninf, 0.0, 1.0, 2.0, ninf, ninf, ninf]] * 2, dtype=np.float32)
+    out = oracle.verify_round(st, zd, zt2, [0], [0.5, 0.5], [0.9])
+    assert out["dist"][0] == 1.0 and out["rejected"]
+    assert (st.nE.value, st.nA.value, st.nR.value) == (2, 0, 0)
+
+
+def test_match_always_accepts_and_update_flag():
+    V, K = 16, 4
+    r = np.random.default_rng(11)
+    st = oracle.SequenceState(capacity=64)
+    zd = r.normal(size=(K, V)).astype(np.float32)
+    zt = r.normal(size=(K + 1, V)).astype(np.float32)
+    ut = r.random(K + 1).astype(np.float32)
+    y = [oracle.inv_cdf(oracle.softmax(zt[i].astype(np.float64))[0], ut[i])[0] for i in range(K + 1)]
+    out = oracle.verify_round(st, zd, zt, y[:K], ut, np.ones(K, dtype=np.float32) * 0.999,
+                              update=False)
+    assert out["accept_len"] == K and np.all(out["p_acc"] == 0.0)
+    assert (st.nE.value, st.nA.value, st.nR.value) == (0, 0, 0)       # update=False leaves state
+    out = oracle.verify_round(st, zd, zt, y[:K], ut, np.ones(K, dtype=np.float32) * 0.999)
+    assert st.nA.value == K and list(out["y"]) == y
+
+
+def test_in_round_appends_feed_later_candidates():
+    """Candidate i sees the accepted distances d_1..d_{i-1} of the same round."""
+    V, K = 16, 3
+    r = np.random.default_rng(5)
+    st = oracle.SequenceState(capacity=64)
+    st.LA[:2] = [0.30, 0.34]
+    st.nA.value = 2
+    st.LR[:3] = [0.6, 0.7, 0.8]
+    st.nR.value = 3
+    zd = r.normal(size=(K, V)).astype(np.float32)
+    zt = (zd + 0.7 * r.normal(size=(K, V))).astype(np.float32)
+    zt = np.concatenate([zt, zd[:1]])
+    ut = r.random(K + 1).astype(np.float32)
+    y = [oracle.inv_cdf(oracle.softmax(zt[i].astype(np.float64))[0], ut[i])[0] for i in range(K)]
+    out = oracle.verify_round(st, zd, zt, y, ut, np.full(K, 0.5, dtype=np.float32), update=False)
+    d = out["dist"]
+    for i in range(K):
+        want = oracle.accept_prob(np.concatenate([[0.30, 0.34], d[:i]]), [0.6, 0.7, 0.8], d[i])
+        stale = oracle.accept_prob([0.30, 0.34], [0.6, 0.7, 0.8], d[i])
+        assert abs(out["p_acc"][i] - want) < 1e-15
+        if i > 0:
+            assert abs(want - stale) > 1e-6
+
+
+def test_reject_rule_threshold_variant():
+    st = oracle.SequenceState(capacity=64, reject_rule=1)
+    st.LA[:3] = [0.1, 0.2, 0.3]
+    st.nA.value = 3
+    st.LR[:3] = [0.7, 0.8, 0.9]
+    st.nR.value = 3
+    z = np.array([[0.0, 0.2, -0.1, 0.05]], dtype=np.float32)
+    zt = np.array([[0.1, 0.1, -0.1, 0.0]] * 2, dtype=np.float32)
+    y0 = oracle.inv_cdf(oracle.softmax(zt[0].astype(np.float64))[0], 0.5)[0]
+    out = oracle.verify_round(st, z, zt, [(y0 + 1) % 4], [0.5, 0.5], [0.999])
+    assert out["p_acc"][0] > 0.5 and out["accept_len"] == 1     # small d: accepted although u is large
+
+
+# ------------------------------------------------------------------ vanilla mode
+
+def logits_of(p):
+    with np.errstate(divide="ignore"):
+        return np.log(np.asarray(p, dtype=np.float64)).astype(np.float32)
+
+
+def test_vanilla_golden_alpha_and_residual(golden):
+    c = golden["vanilla_reversed"]
+    p, q = np.array(c["p"]), np.array(c["q"])
+    zt = np.stack([logits_of(p), logits_of(p)])
+    zd = logits_of(q)[None]
+    for x in range(4):
+        out = oracle.vanilla_round(zd, zt, [x], [0.9999], 0.1)
+        assert abs(out["alpha"][0] - c["expect"]["alpha"][x]) < 1e-6
+    # rejected (u_accept above alpha): the resample follows the residual [0,0,1/4,3/4]
+    for ur, want in [(0.1, 2), (0.24, 2), (0.26, 3), (0.9, 3)]:
+        out = oracle.vanilla_round(zd, zt, [0], [0.5], ur)
+        assert out["accept_len"] == 0 and out["next_token"] == want
+    # accepted everywhere: bonus row sampled with u_resample
+    out = oracle.vanilla_round(zd, zt, [3], [0.5], 0.35)
+    assert out["accept_len"] == 1 and out["next_token"] == 2
+
+
+def test_vanilla_output_law_is_target_distribution():
+    """Leviathan's identity: accept/resample reproduces p_t exactly (V=4 enumeration)."""
+    r = np.random.default_rng(21)
+    N = 120
+    grid = (np.arange(N) + 0.5) / N
+    for _ in range(2):
+        p, q = rand_dist(4), rand_dist(4)
+        zt = np.stack([logits_of(p), logits_of(p)])
+        zd = logits_of(q)[None]
+        pp = oracle.softmax(zt[0].astype(np.float64))[0]
+        qq = oracle.softmax(zd[0].astype(np.float64))[0]
+        law = np.zeros(4)
+        for x in range(4):
+            for ua in grid:
+                acc = oracle.vanilla_round(zd, zt, [x], [ua], 0.5)
+                if acc["accept_len"] == 1:
+                    law[x] += qq[x] / N
+                else:
+                    for ur in grid:
+                        tok = oracle.vanilla_round(zd, zt, [x], [ua], ur)["next_token"]
+                        law[tok] += qq[x] / (N * N)
+        assert np.abs(law - pp).max() < 2.5 / N
+
+
+def test_vanilla_first_rejection_prefix():
+    V, K = 8, 4
+    r = np.random.default_rng(2)
+    zd = r.normal(size=(K, V)).astype(np.float32)
+    zt = np.concatenate([zd, zd[:1]])            # identical rows: alpha == 1 everywhere
+    out = oracle.vanilla_round(zd, zt, [1, 2, 3, 4], [0.999] * K, 0.3)
+    assert out["accept_len"] == K and np.all(out["alpha"] == 1.0)
+    zt2 = zt.copy()
+    zt2[2, 3] -= 20.0                            # token 3 at position 2 becomes very unlikely
+    out = oracle.vanilla_round(zd, zt2, [1, 2, 3, 4], [0.5] * K, 0.3)
+    assert out["accept_len"] == 2 and out["next_token"] != 3 and np.isnan(out["alpha"][3])
