@@ -1,0 +1,450 @@
+// C ABI of the AdaSD hot path (see include/adasd.h): context management, argument
+// validation and kernel launches.  No torch types, no CPU fallback: without a CUDA
+// device every call fails with ADASD_ERR_CUDA.
+#include <cuda_runtime.h>
+
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "adasd_rows.cuh"
+
+using namespace adasd;
+
+struct adasd_ctx {
+    adasd_config cfg;
+    State st;
+    Scratch sc;
+    std::vector<void*> allocs;
+    int sm_count;
+};
+
+namespace {
+
+#define CUDA_TRY(expr)                         \
+    do {                                       \
+        cudaError_t e__ = (expr);              \
+        if (e__ != cudaSuccess) return ADASD_ERR_CUDA; \
+    } while (0)
+
+template <typename T>
+int dev_alloc(adasd_ctx* c, T** p, size_t n) {
+    void* q = nullptr;
+    if (cudaMalloc(&q, n * sizeof(T)) != cudaSuccess) return ADASD_ERR_CUDA;
+    if (cudaMemset(q, 0, n * sizeof(T)) != cudaSuccess) return ADASD_ERR_CUDA;
+    c->allocs.push_back(q);
+    *p = static_cast<T*>(q);
+    return ADASD_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline size_t elt_size(int dtype) { return dtype == ADASD_BF16 ? 2 : 4; }
+
+// Rows can take 16-byte loads when the base and every stride are 16-byte multiples.
+inline bool vec_ok(const void* base, int dtype, std::initializer_list<long long> strides) {
+    if (!aligned16(base)) return false;
+    for (long long s : strides)
+        if ((s * (long long)elt_size(dtype)) % 16 != 0) return false;
+    return true;
+}
+
+int pick_cluster(const adasd_ctx* c, long long rows) {
+    if (c->cfg.cluster_size > 0) return c->cfg.cluster_size;
+    const long long want = 2LL * c->sm_count;
+    for (int cs = 1; cs <= kMaxCluster; cs *= 2)
+        if (rows * cs >= want) return cs;
+    return kMaxCluster;
+}
+
+template <typename P>
+int launch_cluster(void (*kernel)(P), const P& params, long long clusters, int cs,
+                   cudaStream_t stream) {
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    lc.gridDim = dim3((unsigned)(clusters * cs), 1, 1);
+    lc.blockDim = dim3(kThreads, 1, 1);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&lc, kernel, params));
+    return ADASD_OK;
+}
+
+int check_strides(const adasd_ctx* c, long long seq, long long row) {
+    if (row < c->cfg.V || seq < 0) return ADASD_ERR_SHAPE;
+    return ADASD_OK;
+}
+
+int fill_verify_params(adasd_ctx* ctx, VerifyParams& p, const void* zd, const void* zt,
+                       int64_t d_seq, int64_t d_row, int64_t t_seq, int64_t t_row,
+                       const int32_t* x, const int32_t* draft_len) {
+    if (!ctx || !zd || !zt || !x) return ADASD_ERR_NULL;
+    int rc;
+    if ((rc = check_strides(ctx, d_seq, d_row)) != ADASD_OK) return rc;
+    if ((rc = check_strides(ctx, t_seq, t_row)) != ADASD_OK) return rc;
+    memset(&p, 0, sizeof(p));
+    p.zd = zd;
+    p.zt = zt;
+    p.d_seq = d_seq;
+    p.d_row = d_row;
+    p.t_seq = t_seq;
+    p.t_row = t_row;
+    p.x = x;
+    p.draft_len = draft_len;
+    p.sc = ctx->sc;
+    p.st = ctx->st;
+    p.B = ctx->cfg.B;
+    p.V = ctx->cfg.V;
+    p.Kmax = ctx->cfg.Kmax;
+    p.tail.Kmax = ctx->cfg.Kmax;
+    p.tail.min_samples = ctx->cfg.min_kde_samples;
+    p.tail.bw_rule = ctx->cfg.kde_bandwidth;
+    p.tail.reject_rule = ctx->cfg.reject_rule;
+    p.tail.update = 0;
+    return ADASD_OK;
+}
+
+template <int MODE>
+int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
+    const long long positions = (long long)p.B * (p.Kmax + 1);
+    const int cs = pick_cluster(ctx, positions);
+    const bool vec = vec_ok(p.zd, ctx->cfg.dtype, {p.d_seq, p.d_row}) &&
+                     vec_ok(p.zt, ctx->cfg.dtype, {p.t_seq, p.t_row});
+    if (ctx->cfg.dtype == ADASD_BF16) {
+        return vec ? launch_cluster(verify_kernel<__nv_bfloat16, true, MODE>, p, positions, cs, stream)
+                   : launch_cluster(verify_kernel<__nv_bfloat16, false, MODE>, p, positions, cs, stream);
+    }
+    return vec ? launch_cluster(verify_kernel<float, true, MODE>, p, positions, cs, stream)
+               : launch_cluster(verify_kernel<float, false, MODE>, p, positions, cs, stream);
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        if (ok && prev >= 0) {
+            int cur = -1;
+            if (cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+        }
+    }
+};
+
+constexpr size_t kExportHeader = 24;
+
+}  // namespace
+
+extern "C" {
+
+int adasd_create(adasd_ctx** out, const adasd_config* cfg) {
+    if (!out || !cfg) return ADASD_ERR_NULL;
+    *out = nullptr;
+    if (cfg->B < 1 || cfg->V < 1 || cfg->Kmax < 1 || cfg->Kmax > ADASD_KMAX_LIMIT ||
+        cfg->list_capacity < 1)
+        return ADASD_ERR_SHAPE;
+    if ((long long)cfg->B * (cfg->Kmax + 1) > 0x3FFFFFFFLL) return ADASD_ERR_SHAPE;
+    if (cfg->dtype != ADASD_BF16 && cfg->dtype != ADASD_FP32) return ADASD_ERR_DTYPE;
+    if (cfg->kde_bandwidth < 0 || cfg->kde_bandwidth > 1 || cfg->reject_rule < 0 ||
+        cfg->reject_rule > 1)
+        return ADASD_ERR_DTYPE;
+    if (cfg->cluster_size != 0 && cfg->cluster_size != 1 && cfg->cluster_size != 2 &&
+        cfg->cluster_size != 4 && cfg->cluster_size != 8)
+        return ADASD_ERR_SHAPE;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev)
+        return ADASD_ERR_CUDA;
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return ADASD_ERR_CUDA;
+
+    adasd_ctx* c = new (std::nothrow) adasd_ctx();
+    if (!c) return ADASD_ERR_CUDA;
+    c->cfg = *cfg;
+    if (c->cfg.min_kde_samples < 2) c->cfg.min_kde_samples = 2;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) {
+        delete c;
+        return ADASD_ERR_CUDA;
+    }
+    c->sm_count = prop.multiProcessorCount;
+    memset(&c->st, 0, sizeof(c->st));
+    memset(&c->sc, 0, sizeof(c->sc));
+
+    const size_t B = (size_t)cfg->B, K = (size_t)cfg->Kmax, cap = (size_t)cfg->list_capacity;
+    int rc = ADASD_OK;
+    State& s = c->st;
+    Scratch& t = c->sc;
+    s.cap = cfg->list_capacity;
+#define ALLOC(ptr, n)                                        \
+    if (rc == ADASD_OK) rc = dev_alloc(c, &(ptr), (size_t)(n))
+    ALLOC(s.T_G, B);
+    ALLOC(s.sumE, B);
+    ALLOC(s.nE, B);
+    ALLOC(s.nA, B);
+    ALLOC(s.nR, B);
+    ALLOC(s.sumA, B);
+    ALLOC(s.sumA2, B);
+    ALLOC(s.sumR, B);
+    ALLOC(s.sumR2, B);
+    ALLOC(s.LE, B * cap);
+    ALLOC(s.LA, B * cap);
+    ALLOC(s.LR, B * cap);
+    ALLOC(s.status, 1);
+    ALLOC(t.H_d, B * K);
+    ALLOC(t.H_t, B * (K + 1));
+    ALLOC(t.lse_d, B * K);
+    ALLOC(t.lse_t, B * (K + 1));
+    ALLOC(t.jsd, B * K);
+    ALLOC(t.dist, B * K);
+    ALLOC(t.p_acc, B * K);
+    ALLOC(t.y, B * (K + 1));
+    ALLOC(t.van_flag, B * K);
+    ALLOC(t.van_tok, B * (K + 1));
+    ALLOC(t.ticket, B);
+#undef ALLOC
+    if (rc == ADASD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ADASD_ERR_CUDA;
+    if (rc != ADASD_OK) {
+        for (void* q : c->allocs) cudaFree(q);
+        delete c;
+        return rc;
+    }
+    *out = c;
+    return ADASD_OK;
+}
+
+int adasd_destroy(adasd_ctx* ctx) {
+    if (!ctx) return ADASD_ERR_NULL;
+    DeviceGuard guard(ctx->cfg.device);
+    int rc = ADASD_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) rc = ADASD_ERR_CUDA;
+    for (void* q : ctx->allocs)
+        if (cudaFree(q) != cudaSuccess) rc = ADASD_ERR_CUDA;
+    delete ctx;
+    return rc;
+}
+
+int adasd_reset(adasd_ctx* ctx, const int32_t* seq_ids_dev, int32_t n, void* stream) {
+    if (!ctx) return ADASD_ERR_NULL;
+    if (!seq_ids_dev) n = ctx->cfg.B;
+    if (n < 0) return ADASD_ERR_SHAPE;
+    if (n == 0) return ADASD_OK;
+    reset_kernel<<<(n + 127) / 128, 128, 0, (cudaStream_t)stream>>>(ctx->st, seq_ids_dev, n,
+                                                                    ctx->cfg.B);
+    CUDA_TRY(cudaGetLastError());
+    return ADASD_OK;
+}
+
+int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stride,
+                        const float* u_dev, uint8_t* active_inout_dev, float* H_out_dev,
+                        float* lse_out_dev, int32_t* token_out_dev, uint8_t* stop_out_dev,
+                        int32_t* draft_len_inout_dev, void* stream) {
+    if (!ctx || !logits_dev || !H_out_dev) return ADASD_ERR_NULL;
+    if ((u_dev == nullptr) != (token_out_dev == nullptr)) return ADASD_ERR_NULL;
+    if (row_stride < ctx->cfg.V) return ADASD_ERR_SHAPE;
+    DraftParams p;
+    memset(&p, 0, sizeof(p));
+    p.z = logits_dev;
+    p.row_stride = row_stride;
+    p.u = u_dev;
+    p.active = active_inout_dev;
+    p.H_out = H_out_dev;
+    p.lse_out = lse_out_dev;
+    p.token_out = token_out_dev;
+    p.stop_out = stop_out_dev;
+    p.draft_len = draft_len_inout_dev;
+    p.st = ctx->st;
+    p.B = ctx->cfg.B;
+    p.V = ctx->cfg.V;
+    const int cs = pick_cluster(ctx, p.B);
+    const bool vec = vec_ok(logits_dev, ctx->cfg.dtype, {row_stride});
+    cudaStream_t st = (cudaStream_t)stream;
+    if (ctx->cfg.dtype == ADASD_BF16)
+        return vec ? launch_cluster(draft_kernel<__nv_bfloat16, true>, p, p.B, cs, st)
+                   : launch_cluster(draft_kernel<__nv_bfloat16, false>, p, p.B, cs, st);
+    return vec ? launch_cluster(draft_kernel<float, true>, p, p.B, cs, st)
+               : launch_cluster(draft_kernel<float, false>, p, p.B, cs, st);
+}
+
+int adasd_verify(adasd_ctx* ctx, const void* draft_logits_dev, const void* target_logits_dev,
+                 int64_t d_seq_stride, int64_t d_row_stride, int64_t t_seq_stride,
+                 int64_t t_row_stride, const int32_t* draft_tokens_dev,
+                 const int32_t* draft_len_dev, const float* u_target_dev,
+                 const float* u_accept_dev, int32_t* accept_len_dev, int32_t* next_token_dev,
+                 const adasd_round_record* record, uint32_t flags, void* stream) {
+    VerifyParams p;
+    int rc = fill_verify_params(ctx, p, draft_logits_dev, target_logits_dev, d_seq_stride,
+                                d_row_stride, t_seq_stride, t_row_stride, draft_tokens_dev,
+                                draft_len_dev);
+    if (rc != ADASD_OK) return rc;
+    if (!u_target_dev || !u_accept_dev || !accept_len_dev || !next_token_dev)
+        return ADASD_ERR_NULL;
+    if (flags & ~ADASD_FUSE_UPDATE) return ADASD_ERR_SHAPE;
+    p.u_target = u_target_dev;
+    p.u_accept = u_accept_dev;
+    p.accept_len = accept_len_dev;
+    p.next_token = next_token_dev;
+    if (record) p.user = *record;
+    p.tail.update = (flags & ADASD_FUSE_UPDATE) ? 1u : 0u;
+    return launch_verify<MODE_ADASD>(ctx, p, (cudaStream_t)stream);
+}
+
+int adasd_update_thresholds(adasd_ctx* ctx, const adasd_round_record* record, void* stream) {
+    if (!ctx || !record) return ADASD_ERR_NULL;
+    if (!record->H_d || !record->dist || !record->draft_len || !record->accept_len ||
+        !record->rejected)
+        return ADASD_ERR_NULL;
+    const int B = ctx->cfg.B;
+    update_kernel<<<(B + 127) / 128, 128, 0, (cudaStream_t)stream>>>(ctx->st, *record, B,
+                                                                     ctx->cfg.Kmax);
+    CUDA_TRY(cudaGetLastError());
+    return ADASD_OK;
+}
+
+int adasd_vanilla_verify(adasd_ctx* ctx, const void* draft_logits_dev,
+                         const void* target_logits_dev, int64_t d_seq_stride,
+                         int64_t d_row_stride, int64_t t_seq_stride, int64_t t_row_stride,
+                         const int32_t* draft_tokens_dev, const int32_t* draft_len_dev,
+                         const float* u_accept_dev, const float* u_resample_dev,
+                         int32_t* accept_len_dev, int32_t* next_token_dev, float* alpha_out_dev,
+                         void* stream) {
+    VerifyParams p;
+    int rc = fill_verify_params(ctx, p, draft_logits_dev, target_logits_dev, d_seq_stride,
+                                d_row_stride, t_seq_stride, t_row_stride, draft_tokens_dev,
+                                draft_len_dev);
+    if (rc != ADASD_OK) return rc;
+    if (!u_accept_dev || !u_resample_dev || !accept_len_dev || !next_token_dev)
+        return ADASD_ERR_NULL;
+    p.u_accept = u_accept_dev;
+    p.u_resample = u_resample_dev;
+    p.accept_len = accept_len_dev;
+    p.next_token = next_token_dev;
+    p.alpha_out = alpha_out_dev;
+    return launch_verify<MODE_VANILLA>(ctx, p, (cudaStream_t)stream);
+}
+
+int adasd_get_thresholds(adasd_ctx* ctx, float* T_G_dev, int32_t* nE_dev, int32_t* nA_dev,
+                         int32_t* nR_dev, void* stream) {
+    if (!ctx) return ADASD_ERR_NULL;
+    const int B = ctx->cfg.B;
+    get_thresholds_kernel<<<(B + 127) / 128, 128, 0, (cudaStream_t)stream>>>(
+        ctx->st, T_G_dev, nE_dev, nA_dev, nR_dev, B);
+    CUDA_TRY(cudaGetLastError());
+    return ADASD_OK;
+}
+
+int adasd_state_export(adasd_ctx* ctx, int32_t seq, void* host_buf, size_t* bytes) {
+    if (!ctx || !bytes) return ADASD_ERR_NULL;
+    if (seq < 0 || seq >= ctx->cfg.B) return ADASD_ERR_SHAPE;
+    DeviceGuard guard(ctx->cfg.device);
+    CUDA_TRY(cudaDeviceSynchronize());
+    const State& s = ctx->st;
+    int32_t n[3];
+    float tg;
+    CUDA_TRY(cudaMemcpy(&n[0], s.nE + seq, 4, cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemcpy(&n[1], s.nA + seq, 4, cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemcpy(&n[2], s.nR + seq, 4, cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemcpy(&tg, s.T_G + seq, 4, cudaMemcpyDeviceToHost));
+    if (n[0] > s.cap) n[0] = s.cap;   // entropies beyond the capacity were only summed
+    const size_t need = kExportHeader + 4 * ((size_t)n[0] + n[1] + n[2]);
+    if (!host_buf) {
+        *bytes = need;
+        return ADASD_OK;
+    }
+    if (*bytes < need) {
+        *bytes = need;
+        return ADASD_ERR_CAPACITY;
+    }
+    char* o = static_cast<char*>(host_buf);
+    int32_t hdr[4] = {n[0], n[1], n[2], 0};
+    float fh[2] = {tg, 0.f};
+    memcpy(o, hdr, 16);
+    memcpy(o + 16, fh, 8);
+    o += kExportHeader;
+    const float* lists[3] = {s.LE, s.LA, s.LR};
+    for (int k = 0; k < 3; ++k) {
+        if (n[k] > 0)
+            CUDA_TRY(cudaMemcpy(o, lists[k] + (size_t)seq * s.cap, 4 * (size_t)n[k],
+                                cudaMemcpyDeviceToHost));
+        o += 4 * (size_t)n[k];
+    }
+    *bytes = need;
+    return ADASD_OK;
+}
+
+int adasd_state_import(adasd_ctx* ctx, int32_t seq, const void* host_buf, size_t bytes) {
+    if (!ctx || !host_buf) return ADASD_ERR_NULL;
+    if (seq < 0 || seq >= ctx->cfg.B || bytes < kExportHeader) return ADASD_ERR_SHAPE;
+    const char* in = static_cast<const char*>(host_buf);
+    int32_t hdr[4];
+    float fh[2];
+    memcpy(hdr, in, 16);
+    memcpy(fh, in + 16, 8);
+    const State& s = ctx->st;
+    for (int k = 0; k < 3; ++k)
+        if (hdr[k] < 0 || hdr[k] > s.cap) return ADASD_ERR_CAPACITY;
+    if (bytes < kExportHeader + 4 * ((size_t)hdr[0] + hdr[1] + hdr[2])) return ADASD_ERR_SHAPE;
+    DeviceGuard guard(ctx->cfg.device);
+    CUDA_TRY(cudaDeviceSynchronize());
+    const float* src = reinterpret_cast<const float*>(in + kExportHeader);
+    float* lists[3] = {s.LE, s.LA, s.LR};
+    double sums[3] = {0, 0, 0}, sums2[3] = {0, 0, 0};
+    for (int k = 0; k < 3; ++k) {
+        for (int j = 0; j < hdr[k]; ++j) {
+            float v;
+            memcpy(&v, src + j, 4);
+            sums[k] += (double)v;
+            sums2[k] += (double)v * (double)v;
+        }
+        if (hdr[k] > 0)
+            CUDA_TRY(cudaMemcpy(lists[k] + (size_t)seq * s.cap, src, 4 * (size_t)hdr[k],
+                                cudaMemcpyHostToDevice));
+        src += hdr[k];
+    }
+    float tg = hdr[0] > 0 ? (float)(sums[0] / (double)hdr[0]) : fh[0];
+    CUDA_TRY(cudaMemcpy(s.nE + seq, &hdr[0], 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.nA + seq, &hdr[1], 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.nR + seq, &hdr[2], 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.T_G + seq, &tg, 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.sumE + seq, &sums[0], 8, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.sumA + seq, &sums[1], 8, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.sumA2 + seq, &sums2[1], 8, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.sumR + seq, &sums[2], 8, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(s.sumR2 + seq, &sums2[2], 8, cudaMemcpyHostToDevice));
+    return ADASD_OK;
+}
+
+int adasd_status(adasd_ctx* ctx, uint32_t* status_out) {
+    if (!ctx || !status_out) return ADASD_ERR_NULL;
+    DeviceGuard guard(ctx->cfg.device);
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(status_out, ctx->st.status, 4, cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemset(ctx->st.status, 0, 4));
+    return ADASD_OK;
+}
+
+const char* adasd_strerror(int code) {
+    switch (code) {
+        case ADASD_OK: return "ok";
+        case ADASD_ERR_NULL: return "a required pointer is NULL";
+        case ADASD_ERR_ALIGN: return "pointer not aligned as required";
+        case ADASD_ERR_SHAPE: return "size, stride or window out of range";
+        case ADASD_ERR_DTYPE: return "unknown dtype or rule";
+        case ADASD_ERR_CAPACITY: return "size beyond a stated maximum";
+        case ADASD_ERR_TIMEOUT: return "a bounded device wait expired";
+        case ADASD_ERR_CUDA: return "a CUDA runtime call failed";
+        case ADASD_ERR_NAN: return "a row held NaN or no finite logit";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -152,6 +152,26 @@ def uniforms_cpu(seed: int, substream: int, round_: int, B: int, n: int) -> np.n
     return out
 
 
+def round_uniforms_cpu(wl: "Workload", round_: int) -> dict:
+    """All uniforms of one round, float32.
+
+    draft [B,K], target [B,K+1], accept [B,K], vanilla_accept [B,K], resample [B].
+    Common random numbers: target[:, i] == draft[:, i] for i < K, so that the draft
+    token x_i = invCDF(q_i, u) and the target sample y_i = invCDF(p_i, u) agree when
+    p_i and q_i are close - the stand-in for a real draft model agreeing with its
+    target.  With independent uniforms two samples from a 128k-token vocabulary
+    almost never coincide and every round would end at its first candidate.
+    """
+    B, K = wl.B, wl.K
+    d = uniforms_cpu(wl.seed, U_DRAFT, round_, B, K)
+    t = uniforms_cpu(wl.seed, U_TARGET, round_, B, K + 1)
+    t[:, :K] = d
+    return dict(draft=d, target=t,
+                accept=uniforms_cpu(wl.seed, U_ACCEPT, round_, B, K),
+                vanilla_accept=uniforms_cpu(wl.seed, U_VANILLA_ACCEPT, round_, B, K),
+                resample=uniforms_cpu(wl.seed, U_RESAMPLE, round_, B, 1)[:, 0].copy())
+
+
 # ----------------------------------------------------------------------------- workloads
 
 @dataclass(frozen=True)
@@ -266,6 +286,24 @@ class GpuSynth:
             self._stream())
         if rc != 0:
             raise RuntimeError(f"synth_uniforms_gpu failed with CUDA error {rc}")
+
+    def round_uniforms(self, round_: int, out: dict, use_round_dev: bool = False) -> None:
+        """Device twin of round_uniforms_cpu: fills out['draft'|'target'|'accept'|
+        'vanilla_accept'|'resample'] (float32 tensors of the shapes given there)."""
+        K = self.wl.K
+        self.uniforms(U_DRAFT, round_, out["draft"], use_round_dev)
+        self.uniforms(U_TARGET, round_, out["target"], use_round_dev)
+        out["target"][:, :K].copy_(out["draft"])
+        self.uniforms(U_ACCEPT, round_, out["accept"], use_round_dev)
+        self.uniforms(U_VANILLA_ACCEPT, round_, out["vanilla_accept"], use_round_dev)
+        self.uniforms(U_RESAMPLE, round_, out["resample"].view(-1, 1), use_round_dev)
+
+    def new_round_uniforms(self) -> dict:
+        t, B, K = self.torch, self.wl.B, self.wl.K
+        f = dict(dtype=t.float32, device=self.device)
+        return dict(draft=t.empty((B, K), **f), target=t.empty((B, K + 1), **f),
+                    accept=t.empty((B, K), **f), vanilla_accept=t.empty((B, K), **f),
+                    resample=t.empty(B, **f))
 
     def advance_round(self, inc: int = 1) -> None:
         rc = self.lib.synth_counter_add_gpu(self.round_dev.data_ptr(), inc, self._stream())

@@ -1,0 +1,359 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the float64
+oracle on the same seeded inputs.  Tolerances: 1e-4 absolute on entropy, log-sum-exp,
+JS divergence/distance, T_G and P(A|d); discrete results exact except at counted
+near-threshold positions (see tests/lockstep.py)."""
+import ctypes
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return torch
+
+
+@pytest.fixture(scope="module")
+def adasd():
+    import paper_2512_11280_b200 as m
+    m.lib()
+    return m
+
+
+def bf16_bits(t):
+    return t.view(__import__("torch").int16).cpu().numpy().view(np.uint16)
+
+
+def raw(t, torch):
+    """Device logits -> the oracle's raw input (bf16 bits or float32)."""
+    return bf16_bits(t) if t.dtype == torch.bfloat16 else t.cpu().numpy()
+
+
+# ------------------------------------------------------------------ generator
+
+def test_generator_host_and_device_rows_are_bit_identical(torch):
+    for name, V in (("C1", 32000), ("C3", 5000)):
+        wl = synth.WORKLOADS[name].scaled(B=3, V=V, rounds=4)
+        gs = synth.GpuSynth(wl)
+        tdt = torch.bfloat16 if wl.dtype == synth.BF16 else torch.float32
+        zd = torch.empty((wl.B, wl.K, V), dtype=tdt, device="cuda")
+        zt = torch.empty((wl.B, wl.K + 1, V), dtype=tdt, device="cuda")
+        for r in (0, 3):
+            gs.draft_rows(r, zd)
+            gs.target_rows(r, zt)
+            hd, ht = synth.host_round(wl, r)
+            assert np.array_equal(raw(zd, torch).reshape(hd.shape), hd)
+            assert np.array_equal(raw(zt, torch).reshape(ht.shape), ht)
+        u = torch.empty((wl.B, 7), dtype=torch.float32, device="cuda")
+        gs.uniforms(synth.U_ACCEPT, 2, u)
+        assert np.array_equal(u.cpu().numpy(), synth.uniforms_cpu(wl.seed, synth.U_ACCEPT, 2, wl.B, 7))
+        # the round counter kept on the device gives the same rows
+        gs.advance_round(3)
+        gs.draft_rows(0, zd, use_round_dev=True)
+        assert np.array_equal(raw(zd, torch).reshape(hd.shape), synth.host_round(wl, 3)[0])
+
+
+# ------------------------------------------------------------------ workloads in lockstep
+
+def run_lockstep(wl, **kw):
+    from tests.lockstep import Lockstep
+    ls = Lockstep(wl, **kw)
+    rep = ls.run()
+    s = rep.summary()
+    print(wl.name, s)
+    assert rep.flips <= max(2, rep.near_threshold), s
+    return rep
+
+
+def test_c1_tiny_fp32_full(torch):
+    rep = run_lockstep(synth.WORKLOADS["C1"])
+    assert rep.rounds == 20 and rep.positions == 20 * 6
+
+
+@pytest.mark.parametrize("V,dtype,cs", [(4, synth.FP32, 1), (64, synth.BF16, 2), (1000, synth.BF16, 4),
+                                        (1003, synth.FP32, 8), (4099, synth.BF16, 8),
+                                        (40000, synth.BF16, 0), (32768 + 8, synth.FP32, 2)])
+def test_small_and_ragged_vocabularies(torch, V, dtype, cs):
+    wl = synth.WORKLOADS["C3"].scaled(name=f"ragged{V}", B=3, K=4, V=V, dtype=dtype, rounds=10)
+    run_lockstep(wl, cluster_size=cs, min_kde_samples=3)
+
+
+def test_c2_single_stream_adaptive_window(torch):
+    wl = synth.WORKLOADS["C2"].scaled(rounds=40)
+    rep = run_lockstep(wl)
+    assert len(rep.window_hist) >= 2          # the stop check produced different windows
+
+
+def test_c3_batched_with_vanilla(torch):
+    wl = synth.WORKLOADS["C3"].scaled(rounds=24)
+    rep = run_lockstep(wl, follow=[0, 13, 31])
+    assert len(rep.accept_hist) >= 2 and len(rep.vanilla_accept_hist) >= 3
+
+
+def test_c4_large_batch_large_vocab_sampled_sequences(torch):
+    wl = synth.WORKLOADS["C4"].scaled(rounds=5)
+    run_lockstep(wl, follow=[0, 77, 127])
+
+
+def test_c5_streaming_adaptive_sampled_sequences(torch):
+    wl = synth.WORKLOADS["C5"].scaled(rounds=10)
+    rep = run_lockstep(wl, follow=[0, 100, 255])
+    assert max(rep.window_hist) <= 16
+
+
+def test_long_history_kde(torch):
+    """Hundreds of rounds on a small vocabulary: long KDE lists, many rejections."""
+    wl = synth.WORKLOADS["C3"].scaled(name="history", B=4, K=8, V=2048, rounds=300, vanilla=False)
+    rep = run_lockstep(wl, check_lists_every=50)
+    assert rep.n_rejections > 20
+
+
+# ------------------------------------------------------------------ crafted edge cases
+
+class Case:
+    """One verify call on hand-made rows, with the oracle's answer beside it."""
+
+    def __init__(self, torch, adasd, zd, zt, x, ut, ua, draft_len=None, dtype=None, **ctx_kw):
+        B, K, V = zd.shape
+        dtype = dtype or torch.float32
+        self.torch, self.B, self.K, self.V = torch, B, K, V
+        self.ctx = adasd.Context(B, V, K, dtype=adasd.ADASD_FP32 if dtype == torch.float32 else adasd.ADASD_BF16,
+                                 list_capacity=256, **ctx_kw)
+        dev = "cuda"
+        self.zd = torch.tensor(zd, dtype=torch.float32).to(dtype).to(dev)
+        self.zt = torch.tensor(zt, dtype=torch.float32).to(dtype).to(dev)
+        self.x = torch.tensor(x, dtype=torch.int32, device=dev)
+        self.ut = torch.tensor(ut, dtype=torch.float32, device=dev)
+        self.ua = torch.tensor(ua, dtype=torch.float32, device=dev)
+        self.dl = None if draft_len is None else torch.tensor(draft_len, dtype=torch.int32, device=dev)
+        self.al = torch.full((B,), -9, dtype=torch.int32, device=dev)
+        self.nt = torch.full((B,), -9, dtype=torch.int32, device=dev)
+        self.rec = self.ctx.new_record()
+
+    def verify(self, fuse=True):
+        self.ctx.verify(self.zd, self.zt, self.x, self.ut, self.ua, self.al, self.nt, draft_len=self.dl,
+                        record=self.rec, fuse_update=fuse)
+        self.torch.cuda.synchronize()
+        return {k: v.cpu().numpy() for k, v in self.rec.items()}
+
+    def oracle_round(self, b, state, update=True):
+        K_t = self.K if self.dl is None else int(self.dl[b])
+        return oracle.verify_round(state, raw(self.zd[b], self.torch), raw(self.zt[b], self.torch),
+                                   self.x[b, :K_t].cpu().numpy(), self.ut[b].cpu().numpy(),
+                                   self.ua[b].cpu().numpy(), K_t=K_t, update=update)
+
+
+def test_identical_disjoint_and_onehot_rows(torch, adasd):
+    V, K = 1000, 4
+    rng = np.random.default_rng(0)
+    ninf = -np.inf
+    zd = rng.normal(size=(1, K, V)).astype(np.float32) * 2
+    zt = rng.normal(size=(1, K + 1, V)).astype(np.float32) * 2
+    zt[0, 0] = zd[0, 0]                                   # identical rows: d == 0 exactly
+    zd[0, 1, : V // 2] = ninf                             # disjoint supports: d == 1 exactly
+    zt[0, 1, V // 2:] = ninf
+    zd[0, 2, :] = ninf                                    # both one-hot on the same token,
+    zt[0, 2, :] = ninf                                    # with different finite values: d == 0
+    zd[0, 2, 17] = 5.0
+    zt[0, 2, 17] = 7.0
+    x = [[3, 600, 17, 5]]
+    c = Case(torch, adasd, zd, zt, x, rng.random((1, K + 1)), np.full((1, K), 0.5))
+    r = c.verify()
+    st = oracle.SequenceState(capacity=64)
+    o = c.oracle_round(0, st)
+    assert r["jsd"][0, 0] == 0.0 and r["dist"][0, 0] == 0.0 and o["dist"][0] == 0.0
+    assert r["dist"][0, 1] == 1.0 and o["dist"][1] == 1.0
+    assert abs(r["jsd"][0, 1] - math.log(2)) < 1e-6
+    assert r["dist"][0, 2] == 0.0 and r["H_d"][0, 2] == 0.0 and r["H_t"][0, 2] == 0.0
+    assert r["y"][0, 2] == 17
+    for k in ("H_d", "jsd", "dist"):
+        assert np.allclose(r[k][0], o[k], atol=TOL), k
+    assert np.allclose(r["H_t"][0], o["H_t"], atol=TOL)
+    assert list(r["y"][0]) == list(o["y"])
+    assert int(c.al[0]) == o["accept_len"] and int(c.nt[0]) == o["next_token"]
+    g = c.ctx.state_export(0)
+    LE, LA, LR = st.lists()
+    assert (len(g["LE"]), len(g["LA"]), len(g["LR"])) == (len(LE), len(LA), len(LR))
+    assert c.ctx.status() == 0
+
+
+def test_entropy_closed_forms_on_device(torch, adasd):
+    for V in (4, 1000, 128256):
+        ctx = adasd.Context(2, V, 1, dtype=adasd.ADASD_FP32, list_capacity=8)
+        z = torch.zeros((2, V), dtype=torch.float32, device="cuda")
+        z[1, :] = -float("inf")
+        z[1, V // 3] = 2.5                                      # one-hot
+        H = torch.zeros(2, device="cuda")
+        lse = torch.zeros(2, device="cuda")
+        tok = torch.zeros(2, dtype=torch.int32, device="cuda")
+        u = torch.tensor([0.5, 0.99], device="cuda")
+        stop = torch.zeros(2, dtype=torch.uint8, device="cuda")
+        ctx.draft_entropy(z, H, u=u, token_out=tok, lse_out=lse, stop_out=stop)
+        torch.cuda.synchronize()
+        assert abs(float(H[0]) - math.log(V)) < TOL and abs(float(lse[0]) - math.log(V)) < TOL
+        assert float(H[1]) == 0.0 and abs(float(lse[1]) - 2.5) < 1e-6
+        assert int(tok[0]) == V // 2 and int(tok[1]) == V // 3
+        assert int(stop[0]) == 1 and int(stop[1]) == 0           # H > T_G = 0 is strict
+
+
+def test_windows_zero_to_kmax_and_inactive_rows(torch, adasd):
+    V, K, B = 3000, 32, 5
+    rng = np.random.default_rng(4)
+    zd = rng.normal(size=(B, K, V)).astype(np.float32) * 3
+    zt = zd[:, :, :] + rng.normal(size=(B, K, V)).astype(np.float32)
+    zt = np.concatenate([zt, rng.normal(size=(B, 1, V)).astype(np.float32)], axis=1)
+    draft_len = [0, 1, 7, 31, 32]
+    x = rng.integers(0, V, size=(B, K))
+    c = Case(torch, adasd, zd, zt, x, rng.random((B, K + 1)), rng.random((B, K)), draft_len=draft_len,
+             dtype=torch.bfloat16)
+    r = c.verify()
+    for b in range(B):
+        st = oracle.SequenceState(capacity=64)
+        o = c.oracle_round(b, st)
+        K_t = draft_len[b]
+        assert int(c.al[b]) == o["accept_len"] and int(c.nt[b]) == o["next_token"], b
+        assert np.allclose(r["dist"][b, :K_t], o["dist"], atol=TOL)
+        assert np.isnan(r["dist"][b, K_t:]).all()                # untouched beyond the window
+        assert list(r["y"][b, : K_t + 1]) == list(o["y"])
+        assert (r["y"][b, K_t + 1:] == -2).all()
+        assert int(r["draft_len"][b]) == K_t
+    assert c.ctx.status() == 0
+
+
+def test_nan_and_all_minus_inf_rows_set_status_not_faults(torch, adasd):
+    V, K = 500, 2
+    rng = np.random.default_rng(5)
+    zd = rng.normal(size=(2, K, V)).astype(np.float32)
+    zt = rng.normal(size=(2, K + 1, V)).astype(np.float32)
+    zd[0, 1, 100] = np.nan
+    zt[1, 0, :] = -np.inf
+    c = Case(torch, adasd, zd, zt, [[1, 2], [3, 4]], rng.random((2, K + 1)), rng.random((2, K)))
+    r = c.verify()
+    assert np.isnan(r["H_d"][0, 1]) and np.isnan(r["jsd"][0, 1])
+    assert np.isnan(r["H_t"][1, 0]) and r["y"][1, 0] == -1
+    assert np.isfinite(r["H_d"][0, 0]) and np.isfinite(r["H_t"][1, 1])
+    assert c.ctx.status() & adasd.STATUS_NAN
+    assert c.ctx.status() == 0                                   # reading clears it
+
+
+def test_fused_update_equals_verify_then_update(torch, adasd):
+    wl = synth.WORKLOADS["C3"].scaled(B=6, K=6, V=4096, rounds=30)
+    gs = synth.GpuSynth(wl)
+    B, K, V = wl.B, wl.K, wl.V
+    zd = torch.empty((B, K, V), dtype=torch.bfloat16, device="cuda")
+    zt = torch.empty((B, K + 1, V), dtype=torch.bfloat16, device="cuda")
+    ctxs = [adasd.Context(B, V, K, list_capacity=512) for _ in range(2)]
+    outs = [[torch.zeros(B, dtype=torch.int32, device="cuda") for _ in range(2)] for _ in range(2)]
+    recs = [c.new_record() for c in ctxs]
+    rng = np.random.default_rng(8)
+    for r in range(wl.rounds):
+        gs.draft_rows(r, zd)
+        gs.target_rows(r, zt)
+        x = torch.tensor(rng.integers(0, V, size=(B, K)), dtype=torch.int32, device="cuda")
+        ut = torch.tensor(rng.random((B, K + 1)), dtype=torch.float32, device="cuda")
+        ua = torch.tensor(rng.random((B, K)), dtype=torch.float32, device="cuda")
+        # make about half of the draft tokens agree with the target sample
+        ctxs[0].verify(zd, zt, x, ut, ua, outs[0][0], outs[0][1], record=recs[0], fuse_update=False)
+        x = torch.where(torch.tensor(rng.random((B, K)) < 0.6, device="cuda"), recs[0]["y"][:, :K], x)
+        ctxs[0].verify(zd, zt, x, ut, ua, outs[0][0], outs[0][1], record=recs[0], fuse_update=True)
+        ctxs[1].verify(zd, zt, x, ut, ua, outs[1][0], outs[1][1], record=recs[1], fuse_update=False)
+        ctxs[1].update_thresholds(recs[1])
+        assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    for b in range(B):
+        a, c = ctxs[0].state_export(b), ctxs[1].state_export(b)
+        assert a["T_G"] == c["T_G"]
+        for k in ("LE", "LA", "LR"):
+            assert np.array_equal(a[k], c[k]), k
+    assert sum(len(ctxs[0].state_export(b)["LR"]) for b in range(B)) > 0
+
+
+def test_state_export_import_reset_roundtrip(torch, adasd):
+    ctx = adasd.Context(3, 100, 4, list_capacity=16)
+    LE, LA, LR = [1.5, 2.5], [0.1, 0.2, 0.3], [0.7, 0.9]
+    ctx.state_import(1, 0.0, LE, LA, LR)
+    g = ctx.state_export(1)
+    assert np.allclose(g["LE"], LE) and np.allclose(g["LA"], LA) and np.allclose(g["LR"], LR)
+    assert abs(g["T_G"] - 2.0) < 1e-7                      # recomputed as mean(L_E^R)
+    T, nE, nA, nR = (t.cpu().numpy() for t in ctx.get_thresholds())
+    assert list(nE) == [0, 2, 0] and list(nA) == [0, 3, 0] and list(nR) == [0, 2, 0]
+    assert abs(T[1] - 2.0) < 1e-7 and T[0] == 0
+    with pytest.raises(adasd.AdasdError):
+        ctx.state_import(1, 0.0, list(range(17)), [], [])   # beyond the capacity
+    with pytest.raises(adasd.AdasdError):
+        ctx.state_export(3)
+    ctx.reset(torch.tensor([1], dtype=torch.int32, device="cuda"))
+    g = ctx.state_export(1)
+    assert g["T_G"] == 0.0 and len(g["LE"]) == len(g["LA"]) == len(g["LR"]) == 0
+
+
+def test_host_detected_errors_launch_nothing(torch, adasd):
+    ctx = adasd.Context(2, 1000, 4)
+    z = torch.zeros((2, 5, 1000), dtype=torch.bfloat16, device="cuda")
+    i = torch.zeros((2, 5), dtype=torch.int32, device="cuda")
+    f = torch.zeros((2, 5), dtype=torch.float32, device="cuda")
+    h = ctx.handle
+    p = lambda t: t.data_ptr()
+    assert adasd.adasd_verify(h, None, p(z), 5000, 1000, 5000, 1000, p(i), None, p(f), p(f), p(i), p(i),
+                              None, 0, None) == -1
+    assert adasd.adasd_verify(h, p(z), p(z), 5000, 999, 5000, 1000, p(i), None, p(f), p(f), p(i), p(i),
+                              None, 0, None) == -3
+    assert adasd.adasd_verify(h, p(z), p(z), 5000, 1000, 5000, 1000, p(i), None, p(f), p(f), p(i), p(i),
+                              None, 8, None) == -3
+    assert adasd.adasd_draft_entropy(h, p(z), 1000, p(f), None, p(f), None, None, None, None, None) == -1
+    assert adasd.adasd_draft_entropy(h, p(z), 10, None, None, p(f), None, None, None, None, None) == -3
+    assert adasd.adasd_vanilla_verify(h, p(z), p(z), 5000, 1000, 5000, 1000, p(i), None, p(f), None,
+                                      p(i), p(i), None, None) == -1
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+
+
+def test_unaligned_rows_take_the_scalar_path(torch, adasd):
+    """Row stride of 1001 bf16 elements: neither base nor stride is 16-byte aligned."""
+    V, K, B = 1001, 3, 2
+    rng = np.random.default_rng(6)
+    zd = rng.normal(size=(B, K, V)).astype(np.float32) * 2
+    zt = np.concatenate([zd + rng.normal(size=(B, K, V)).astype(np.float32) * 0.5,
+                         rng.normal(size=(B, 1, V)).astype(np.float32)], axis=1)
+    c = Case(torch, adasd, zd, zt, rng.integers(0, V, size=(B, K)), rng.random((B, K + 1)),
+             rng.random((B, K)), dtype=torch.bfloat16)
+    assert (c.zd.stride(1) * 2) % 16 != 0
+    r = c.verify()
+    for b in range(B):
+        o = c.oracle_round(b, oracle.SequenceState(capacity=64))
+        for k in ("H_d", "jsd", "dist"):
+            assert np.allclose(r[k][b], o[k], atol=TOL), k
+        assert list(r["y"][b]) == list(o["y"])
+
+
+def test_repeatable_bitwise(torch, adasd):
+    wl = synth.WORKLOADS["C3"].scaled(B=8, K=8, V=128256, rounds=2)
+    gs = synth.GpuSynth(wl)
+    zd = torch.empty((8, 8, wl.V), dtype=torch.bfloat16, device="cuda")
+    zt = torch.empty((8, 9, wl.V), dtype=torch.bfloat16, device="cuda")
+    gs.draft_rows(0, zd)
+    gs.target_rows(0, zt)
+    x = torch.zeros((8, 8), dtype=torch.int32, device="cuda")
+    ut = torch.rand((8, 9), device="cuda")
+    ua = torch.rand((8, 8), device="cuda")
+    res = []
+    for _ in range(2):
+        ctx = adasd.Context(8, wl.V, 8)
+        rec = ctx.new_record()
+        al = torch.zeros(8, dtype=torch.int32, device="cuda")
+        nt = torch.zeros(8, dtype=torch.int32, device="cuda")
+        ctx.verify(zd, zt, x, ut, ua, al, nt, record=rec)
+        torch.cuda.synchronize()
+        res.append({k: v.clone() for k, v in rec.items()})
+    for k in res[0]:
+        a, b = res[0][k], res[1][k]
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32)), k
