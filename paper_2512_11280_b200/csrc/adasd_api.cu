@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "adasd_rows.cuh"
+#include "adasd_staged.cuh"
 
 using namespace adasd;
 
@@ -18,6 +19,10 @@ struct adasd_ctx {
     Scratch sc;
     std::vector<void*> allocs;
     int sm_count;
+    // staged (bulk-copy, persistent cluster) path: 0 = not usable for this V / dtype
+    int staged_iter;          // 16-byte units per lane per row
+    int staged_slice_pad;     // bytes of one CTA's slice of one row, padded
+    int staged_clusters[2];   // resident clusters per mode (AdaSD, vanilla)
 };
 
 namespace {
@@ -78,6 +83,100 @@ int launch_cluster(void (*kernel)(P), const P& params, long long clusters, int c
     return ADASD_OK;
 }
 
+template <int ITER, int MODE>
+int staged_prepare(adasd_ctx* c) {
+    auto kern = staged_verify_kernel<ITER, MODE>;
+    const int smem = 4 * c->staged_slice_pad;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    lc.gridDim = dim3(kSC * 64, 1, 1);
+    lc.blockDim = dim3(kSThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kSC;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &lc) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
+template <int MODE>
+int staged_prepare_iter(adasd_ctx* c) {
+    switch (c->staged_iter) {
+        case 1: return staged_prepare<1, MODE>(c);
+        case 2: return staged_prepare<2, MODE>(c);
+        case 3: return staged_prepare<3, MODE>(c);
+        case 4: return staged_prepare<4, MODE>(c);
+        case 5: return staged_prepare<5, MODE>(c);
+        default: return 0;
+    }
+}
+
+// The staged path needs bf16 rows of a multiple of 8 elements, long enough to give every
+// warp of a cluster work and short enough for the register stash.
+void staged_setup(adasd_ctx* c) {
+    c->staged_iter = 0;
+    c->staged_clusters[0] = c->staged_clusters[1] = 0;
+    const int V = c->cfg.V;
+    if (c->cfg.dtype != ADASD_BF16 || (V & 7) != 0 || V < 8192) return;
+    if (c->cfg.cluster_size != 0 && c->cfg.cluster_size != kSC) return;
+    const int NU = V >> 3;
+    const int per_cta = (NU + kSC - 1) / kSC;
+    const int per_warp = (per_cta + kSW - 1) / kSW + 1;
+    const int iter = (per_warp + 31) / 32;
+    if (iter > kStagedMaxIter) return;
+    c->staged_iter = iter;
+    c->staged_slice_pad = ((per_cta + 1) * 16 + 127) & ~127;
+    c->staged_clusters[0] = staged_prepare_iter<MODE_ADASD>(c);
+    c->staged_clusters[1] = staged_prepare_iter<MODE_VANILLA>(c);
+    if (c->staged_clusters[0] < 1 || c->staged_clusters[1] < 1) c->staged_iter = 0;
+}
+
+template <int ITER, int MODE>
+int staged_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
+    const long long positions = (long long)p.B * (p.Kmax + 1);
+    int ncl = c->staged_clusters[MODE];
+    if (positions < ncl) ncl = (int)positions;
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    lc.gridDim = dim3((unsigned)(ncl * kSC), 1, 1);
+    lc.blockDim = dim3(kSThreads, 1, 1);
+    lc.dynamicSmemBytes = 4 * c->staged_slice_pad;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kSC;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&lc, staged_verify_kernel<ITER, MODE>, p, ncl, c->staged_slice_pad));
+    return ADASD_OK;
+}
+
+template <int MODE>
+int staged_launch_iter(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
+    switch (c->staged_iter) {
+        case 1: return staged_launch<1, MODE>(c, p, stream);
+        case 2: return staged_launch<2, MODE>(c, p, stream);
+        case 3: return staged_launch<3, MODE>(c, p, stream);
+        case 4: return staged_launch<4, MODE>(c, p, stream);
+        case 5: return staged_launch<5, MODE>(c, p, stream);
+        default: return ADASD_ERR_SHAPE;
+    }
+}
+
 int check_strides(const adasd_ctx* c, long long seq, long long row) {
     if (row < c->cfg.V || seq < 0) return ADASD_ERR_SHAPE;
     return ADASD_OK;
@@ -118,6 +217,7 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
     const int cs = pick_cluster(ctx, positions);
     const bool vec = vec_ok(p.zd, ctx->cfg.dtype, {p.d_seq, p.d_row}) &&
                      vec_ok(p.zt, ctx->cfg.dtype, {p.t_seq, p.t_row});
+    if (vec && ctx->staged_iter > 0) return staged_launch_iter<MODE>(ctx, p, stream);
     if (ctx->cfg.dtype == ADASD_BF16) {
         return vec ? launch_cluster(verify_kernel<__nv_bfloat16, true, MODE>, p, positions, cs, stream)
                    : launch_cluster(verify_kernel<__nv_bfloat16, false, MODE>, p, positions, cs, stream);
@@ -212,6 +312,7 @@ int adasd_create(adasd_ctx** out, const adasd_config* cfg) {
     ALLOC(t.van_tok, B * (K + 1));
     ALLOC(t.ticket, B);
 #undef ALLOC
+    if (rc == ADASD_OK) staged_setup(c);
     if (rc == ADASD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ADASD_ERR_CUDA;
     if (rc != ADASD_OK) {
         for (void* q : c->allocs) cudaFree(q);

@@ -172,7 +172,8 @@ def test_identical_disjoint_and_onehot_rows(torch, adasd):
     st = oracle.SequenceState(capacity=64)
     o = c.oracle_round(0, st)
     assert r["jsd"][0, 0] == 0.0 and r["dist"][0, 0] == 0.0 and o["dist"][0] == 0.0
-    assert r["dist"][0, 1] == 1.0 and o["dist"][1] == 1.0
+    # disjoint supports: exactly 1 on the device; the oracle's float64 sum is within rounding of 1
+    assert r["dist"][0, 1] == 1.0 and abs(o["dist"][1] - 1.0) < 1e-12, (r["dist"][0, 1], o["dist"][1])
     assert abs(r["jsd"][0, 1] - math.log(2)) < 1e-6
     assert r["dist"][0, 2] == 0.0 and r["H_d"][0, 2] == 0.0 and r["H_t"][0, 2] == 0.0
     assert r["y"][0, 2] == 17
