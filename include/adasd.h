@@ -60,6 +60,10 @@ extern "C" {
 
 #define ADASD_KMAX_LIMIT 32      /* largest window supported (the paper uses W = 20) */
 
+/* limits of adasd_vanilla_verify_static (its scratch is a fixed array of about 132 KB) */
+#define ADASD_STATIC_MAX_B 1024            /* sequences per call */
+#define ADASD_STATIC_MAX_POSITIONS 16384   /* B * (Kmax + 1) per call */
+
 /* flags of adasd_verify */
 #define ADASD_FUSE_UPDATE 1u     /* run the list appends and the T_G update in the same launch */
 
@@ -170,6 +174,46 @@ int adasd_vanilla_verify(adasd_ctx* ctx, const void* draft_logits_dev,
                          const float* u_accept_dev, const float* u_resample_dev,
                          int32_t* accept_len_dev, int32_t* next_token_dev, float* alpha_out_dev,
                          void* stream);
+
+/*
+ * Vanilla verification for callers that must not allocate device memory.  (The paper has
+ * no counterpart: this is a packaging variant of adasd_vanilla_verify, same inputs, same
+ * outputs, same arithmetic.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a serving engine
+ * that has handed the whole GPU to its own memory pool, in a plugin or callback that is
+ * forbidden to touch the allocator, or in a process that may not grow its footprint after
+ * start-up.  Such a caller cannot use adasd_create(), which allocates the context's
+ * state.  This entry point needs no context: the few words of scratch the kernel uses
+ * between its blocks (per-candidate accept flags, per-position candidate tokens, per-
+ * sequence arrival counters, a status word) live in a fixed array inside the library
+ * image.  It calls neither cudaMalloc nor cudaFree nor any routine that does.
+ *
+ *   B, V, Kmax, dtype   as in adasd_config; B <= ADASD_STATIC_MAX_B and
+ *                       B * (Kmax + 1) <= ADASD_STATIC_MAX_POSITIONS, else
+ *                       ADASD_ERR_CAPACITY is returned and nothing is launched
+ *   logits, strides, draft_tokens_dev, draft_len_dev, u_accept_dev, u_resample_dev,
+ *   accept_len_dev, next_token_dev, alpha_out_dev      as in adasd_vanilla_verify
+ *   status_out_dev      nullable device word: receives the ADASD_STATUS_* bits of this
+ *                       call (cleared first)
+ *
+ * The device used is the calling thread's current device.  The first call on each device
+ * looks up the device address of the scratch array (one cudaGetSymbolAddress, no
+ * allocation); make that first call outside any stream capture.  Every GPU that loads the
+ * library holds the array (about 132 KB) until the process exits.  All calls on a device
+ * share it, and it keeps the previous call's contents: each call clears the counters and
+ * the status word it needs on `stream` before its kernel.  Two calls that overlap on the
+ * same GPU (different streams, different threads) race on the array and give wrong
+ * results: serialise them on one stream.
+ */
+int adasd_vanilla_verify_static(int32_t B, int32_t V, int32_t Kmax, int32_t dtype,
+                                const void* draft_logits_dev, const void* target_logits_dev,
+                                int64_t d_seq_stride, int64_t d_row_stride, int64_t t_seq_stride,
+                                int64_t t_row_stride, const int32_t* draft_tokens_dev,
+                                const int32_t* draft_len_dev, const float* u_accept_dev,
+                                const float* u_resample_dev, int32_t* accept_len_dev,
+                                int32_t* next_token_dev, float* alpha_out_dev,
+                                uint32_t* status_out_dev, void* stream);
 
 /* Copies T_G and the list sizes |L_E^R|, |L_D^A|, |L_D^R| to caller arrays [B] (each nullable). */
 int adasd_get_thresholds(adasd_ctx* ctx, float* T_G_dev, int32_t* nE_dev, int32_t* nA_dev,

@@ -9,7 +9,7 @@ from .binding import (ADASD_BF16, ADASD_FP32, ADASD_FUSE_UPDATE, ADASD_KMAX_LIMI
                       STATUS_NAN, STATUS_TIMEOUT, AdasdConfig, AdasdError, Context, RoundRecord,
                       adasd_create, adasd_destroy, adasd_draft_entropy, adasd_get_thresholds,
                       adasd_reset, adasd_state_export, adasd_state_import, adasd_status,
-                      adasd_strerror, adasd_update_thresholds, adasd_vanilla_verify, adasd_verify,
+                      adasd_strerror, adasd_update_thresholds, adasd_vanilla_verify, adasd_vanilla_verify_static, adasd_verify,
                       lib, library_path)
 from .build import build
 

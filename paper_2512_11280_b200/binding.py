@@ -61,6 +61,8 @@ def lib() -> C.CDLL:
                          U32, P],
         "adasd_update_thresholds": [P, C.POINTER(RoundRecord), P],
         "adasd_vanilla_verify": [P, P, P, I64, I64, I64, I64, P, P, P, P, P, P, P, P],
+        "adasd_vanilla_verify_static": [I32, I32, I32, I32, P, P, I64, I64, I64, I64, P, P, P, P,
+                                        P, P, P, P, P],
         "adasd_get_thresholds": [P, P, P, P, P, P],
         "adasd_state_export": [P, I32, P, C.POINTER(C.c_size_t)],
         "adasd_state_import": [P, I32, P, C.c_size_t],
@@ -126,6 +128,21 @@ def adasd_vanilla_verify(ctx, draft_logits_dev, target_logits_dev, d_seq_stride,
                                       d_row_stride, t_seq_stride, t_row_stride, draft_tokens_dev,
                                       draft_len_dev, u_accept_dev, u_resample_dev, accept_len_dev,
                                       next_token_dev, alpha_out_dev, stream)
+
+
+def adasd_vanilla_verify_static(B, V, Kmax, dtype, draft_logits_dev, target_logits_dev,
+                                d_seq_stride, d_row_stride, t_seq_stride, t_row_stride,
+                                draft_tokens_dev, draft_len_dev, u_accept_dev, u_resample_dev,
+                                accept_len_dev, next_token_dev, alpha_out_dev, status_out_dev,
+                                stream) -> int:
+    """Context-free vanilla verification whose scratch is a fixed array inside the library:
+    for callers that may not allocate device memory.  Same arguments as the C function."""
+    return lib().adasd_vanilla_verify_static(B, V, Kmax, dtype, draft_logits_dev,
+                                             target_logits_dev, d_seq_stride, d_row_stride,
+                                             t_seq_stride, t_row_stride, draft_tokens_dev,
+                                             draft_len_dev, u_accept_dev, u_resample_dev,
+                                             accept_len_dev, next_token_dev, alpha_out_dev,
+                                             status_out_dev, stream)
 
 
 def adasd_get_thresholds(ctx, T_G_dev, nE_dev, nA_dev, nR_dev, stream) -> int:

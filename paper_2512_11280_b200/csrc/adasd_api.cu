@@ -5,6 +5,7 @@
 
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -243,6 +244,47 @@ struct DeviceGuard {
 
 constexpr size_t kExportHeader = 24;
 
+}  // namespace
+
+// ---- allocation-free vanilla verification -------------------------------------------
+// Scratch of adasd_vanilla_verify_static: lives in the library image, one copy per GPU
+// that loads it, shared by every call.  Words: per-candidate accept flags, per-position
+// candidate tokens, per-sequence arrival counters, one status word.
+static __device__ __align__(256) uint32_t g_static_scratch[2 * ADASD_STATIC_MAX_POSITIONS +
+                                                           ADASD_STATIC_MAX_B + 64];
+
+namespace {
+constexpr int kMaxDevices = 64;
+struct StaticSetup {
+    uint32_t* base = nullptr;   // device address of g_static_scratch on this device
+    int sm_count = 0;
+};
+StaticSetup g_static_setup[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Device address of the scratch array on the CURRENT device.  The array's name is only a
+// host-side handle: the address a kernel can use comes from cudaGetSymbolAddress, asked
+// once per device with that device current.
+int static_setup(int dev, StaticSetup& out) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticSetup& s = g_static_setup[dev];
+    if (!s.base) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return ADASD_ERR_CUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return ADASD_ERR_CUDA;
+        }
+        s.sm_count = sms;
+        s.base = static_cast<uint32_t*>(ptr);
+    }
+    out = s;
+    return ADASD_OK;
+}
 }  // namespace
 
 extern "C" {
@@ -531,6 +573,81 @@ int adasd_status(adasd_ctx* ctx, uint32_t* status_out) {
     CUDA_TRY(cudaMemcpy(status_out, ctx->st.status, 4, cudaMemcpyDeviceToHost));
     CUDA_TRY(cudaMemset(ctx->st.status, 0, 4));
     return ADASD_OK;
+}
+
+int adasd_vanilla_verify_static(int32_t B, int32_t V, int32_t Kmax, int32_t dtype,
+                                const void* draft_logits_dev, const void* target_logits_dev,
+                                int64_t d_seq_stride, int64_t d_row_stride, int64_t t_seq_stride,
+                                int64_t t_row_stride, const int32_t* draft_tokens_dev,
+                                const int32_t* draft_len_dev, const float* u_accept_dev,
+                                const float* u_resample_dev, int32_t* accept_len_dev,
+                                int32_t* next_token_dev, float* alpha_out_dev,
+                                uint32_t* status_out_dev, void* stream) {
+    if (!draft_logits_dev || !target_logits_dev || !draft_tokens_dev || !u_accept_dev ||
+        !u_resample_dev || !accept_len_dev || !next_token_dev)
+        return ADASD_ERR_NULL;
+    if (dtype != ADASD_BF16 && dtype != ADASD_FP32) return ADASD_ERR_DTYPE;
+    if (B < 1 || V < 1 || Kmax < 1 || Kmax > ADASD_KMAX_LIMIT) return ADASD_ERR_SHAPE;
+    if (B > ADASD_STATIC_MAX_B || (long long)B * (Kmax + 1) > ADASD_STATIC_MAX_POSITIONS)
+        return ADASD_ERR_CAPACITY;
+    if (d_row_stride < V || t_row_stride < V || d_seq_stride < 0 || t_seq_stride < 0)
+        return ADASD_ERR_SHAPE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return ADASD_ERR_CUDA;
+    }
+    StaticSetup su;
+    int rc = static_setup(dev, su);
+    if (rc != ADASD_OK) return rc;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    uint32_t* flag = su.base;
+    uint32_t* tok = su.base + ADASD_STATIC_MAX_POSITIONS;
+    uint32_t* ticket = su.base + 2 * ADASD_STATIC_MAX_POSITIONS;
+    uint32_t* status = status_out_dev ? status_out_dev : ticket + ADASD_STATIC_MAX_B;
+    // the array keeps whatever the previous call left: counters and status start at zero
+    CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(uint32_t) * (size_t)B, st));
+    CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(uint32_t), st));
+
+    VerifyParams p;
+    memset(&p, 0, sizeof(p));
+    p.zd = draft_logits_dev;
+    p.zt = target_logits_dev;
+    p.d_seq = d_seq_stride;
+    p.d_row = d_row_stride;
+    p.t_seq = t_seq_stride;
+    p.t_row = t_row_stride;
+    p.x = draft_tokens_dev;
+    p.draft_len = draft_len_dev;
+    p.u_accept = u_accept_dev;
+    p.u_resample = u_resample_dev;
+    p.accept_len = accept_len_dev;
+    p.next_token = next_token_dev;
+    p.alpha_out = alpha_out_dev;
+    p.sc.van_flag = reinterpret_cast<int32_t*>(flag);
+    p.sc.van_tok = reinterpret_cast<int32_t*>(tok);
+    p.sc.ticket = ticket;
+    p.st.status = status;
+    p.B = B;
+    p.V = V;
+    p.Kmax = Kmax;
+    p.tail.Kmax = Kmax;
+
+    const long long positions = (long long)B * (Kmax + 1);
+    int cs = kMaxCluster;
+    for (int c = 1; c <= kMaxCluster; c *= 2)
+        if (positions * c >= 2LL * su.sm_count) {
+            cs = c;
+            break;
+        }
+    const bool vec = vec_ok(draft_logits_dev, dtype, {d_seq_stride, d_row_stride}) &&
+                     vec_ok(target_logits_dev, dtype, {t_seq_stride, t_row_stride});
+    if (dtype == ADASD_BF16)
+        return vec ? launch_cluster(verify_kernel<__nv_bfloat16, true, MODE_VANILLA>, p, positions, cs, st)
+                   : launch_cluster(verify_kernel<__nv_bfloat16, false, MODE_VANILLA>, p, positions, cs, st);
+    return vec ? launch_cluster(verify_kernel<float, true, MODE_VANILLA>, p, positions, cs, st)
+               : launch_cluster(verify_kernel<float, false, MODE_VANILLA>, p, positions, cs, st);
 }
 
 const char* adasd_strerror(int code) {
