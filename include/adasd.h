@@ -78,7 +78,7 @@ typedef struct {
     int32_t kde_bandwidth;   /* 0: Silverman factor (3n/4)^(-1/5); 1: Scott n^(-1/5) */
     int32_t reject_rule;     /* 0: Bernoulli, reject iff u >= P(A|d); 1: reject iff P(A|d) < 1/2 */
     int32_t min_kde_samples; /* below this many entries in either list P(A|d) := 0 (>= 2) */
-    int32_t cluster_size;    /* 0 = choose automatically; else 1, 2, 4 or 8 CTAs per row */
+    int32_t cluster_size;    /* 0 = choose automatically; else 1..8 CTAs per row / position */
     int32_t device;          /* CUDA device ordinal */
 } adasd_config;
 

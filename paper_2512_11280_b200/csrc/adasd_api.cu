@@ -3,6 +3,7 @@
 // device every call fails with ADASD_ERR_CUDA.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -10,7 +11,7 @@
 #include <vector>
 
 #include "adasd_rows.cuh"
-#include "adasd_staged.cuh"
+#include "adasd_cluster.cuh"
 
 using namespace adasd;
 
@@ -20,10 +21,12 @@ struct adasd_ctx {
     Scratch sc;
     std::vector<void*> allocs;
     int sm_count;
-    // staged (bulk-copy, persistent cluster) path: 0 = not usable for this V / dtype
-    int staged_iter;          // 16-byte units per lane per row
-    int staged_slice_pad;     // bytes of one CTA's slice of one row, padded
-    int staged_clusters[2];   // resident clusters per mode (AdaSD, vanilla)
+    // streaming cluster kernel: fast_iter == 0 means not usable for this V / dtype
+    int fast_iter;            // iterations per warp and row (template parameter)
+    int fast_cs;              // CTAs per cluster
+    int fast_ncl;             // clusters resident at once (both modes)
+    int fast_smem;            // dynamic shared memory per CTA
+    ClusterGeom fast_geom;
 };
 
 namespace {
@@ -84,22 +87,22 @@ int launch_cluster(void (*kernel)(P), const P& params, long long clusters, int c
     return ADASD_OK;
 }
 
+// ---- streaming cluster kernel: configuration and launch ---------------------------------
 template <int ITER, int MODE>
-int staged_prepare(adasd_ctx* c) {
-    auto kern = staged_verify_kernel<ITER, MODE>;
-    const int smem = 4 * c->staged_slice_pad;
+int fast_occupancy(int cs, int smem) {
+    auto kern = cluster_verify_kernel<ITER, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
-    lc.gridDim = dim3(kSC * 64, 1, 1);
-    lc.blockDim = dim3(kSThreads, 1, 1);
-    lc.dynamicSmemBytes = smem;
+    lc.gridDim = dim3((unsigned)(cs * 64), 1, 1);
+    lc.blockDim = dim3(kCThreads, 1, 1);
+    lc.dynamicSmemBytes = (size_t)smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kSC;
+    attr[0].val.clusterDim.x = (unsigned)cs;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
@@ -112,70 +115,109 @@ int staged_prepare(adasd_ctx* c) {
     return n;
 }
 
-template <int MODE>
-int staged_prepare_iter(adasd_ctx* c) {
-    switch (c->staged_iter) {
-        case 1: return staged_prepare<1, MODE>(c);
-        case 2: return staged_prepare<2, MODE>(c);
-        case 3: return staged_prepare<3, MODE>(c);
-        case 4: return staged_prepare<4, MODE>(c);
-        case 5: return staged_prepare<5, MODE>(c);
-        default: return 0;
+template <int ITER, int MODE>
+int fast_static_smem() {
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, cluster_verify_kernel<ITER, MODE>) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
+    return (int)fa.sharedSizeBytes;
+}
+
+#define ADASD_ITER_SWITCH(iter, CALL, fail)  \
+    switch (iter) {                          \
+        case 1: return CALL(1);              \
+        case 2: return CALL(2);              \
+        case 3: return CALL(3);              \
+        case 4: return CALL(4);              \
+        case 5: return CALL(5);              \
+        case 6: return CALL(6);              \
+        case 7: return CALL(7);              \
+        case 8: return CALL(8);              \
+        case 9: return CALL(9);              \
+        case 10: return CALL(10);            \
+        default: return fail;                \
+    }
+
+int fast_occupancy_iter(int iter, int cs, int smem) {
+#define CALL(I) std::min(fast_occupancy<I, MODE_ADASD>(cs, smem), fast_occupancy<I, MODE_VANILLA>(cs, smem))
+    ADASD_ITER_SWITCH(iter, CALL, 0)
+#undef CALL
+}
+int fast_static_smem_iter(int iter) {
+#define CALL(I) std::max(fast_static_smem<I, MODE_ADASD>(), fast_static_smem<I, MODE_VANILLA>())
+    ADASD_ITER_SWITCH(iter, CALL, -1)
+#undef CALL
+}
+
+// Chooses the cluster size that covers the most SMs among those whose per-CTA slice fits on
+// chip: the kept 2^t values (registers first, shared memory for the rest) plus a ring of at
+// least one position.  bf16 rows of a multiple of 8 elements only.
+void fast_setup(adasd_ctx* c, size_t smem_optin) {
+    c->fast_iter = 0;
+    const int V = c->cfg.V;
+    if (c->cfg.dtype != ADASD_BF16 || (V & 7) != 0 || V < 8192) return;
+    const int NU = V >> 3;
+    int best_score = 0;
+    for (int cs = kCMaxCluster; cs >= 1; --cs) {
+        if (c->cfg.cluster_size != 0 && c->cfg.cluster_size != cs) continue;
+        const int ncu = (NU + cs - 1) / cs, nwi = (ncu + 31) / 32;
+        const int I_lo = nwi / kCW, rem = nwi % kCW, iter = I_lo + (rem ? 1 : 0);
+        if (iter < 1 || iter > kCMaxIter) continue;
+        const int KR = std::min(iter, kCRegIter);
+        int stash_slots = 0;
+        if (iter > KR) stash_slots = (iter - 1 - KR) * kCW + ((iter - 1 < I_lo) ? kCW : rem);
+        const int stash_bytes = stash_slots * kCSlotBytes;
+        const int st = fast_static_smem_iter(iter);
+        if (st < 0) continue;
+        const int avail = (int)smem_optin - st - stash_bytes - 1024;
+        const int n_stg = (iter + 1) / 2;
+        int NS = std::min({kCMaxSlots, avail / (kCW * kCSlotBytes), 2 * n_stg});
+        if (NS < n_stg) continue;
+        const int smem = NS * kCW * kCSlotBytes + stash_bytes;
+        const int ncl = fast_occupancy_iter(iter, cs, smem);
+        const int score = ncl * cs;
+        if (score > best_score) {
+            best_score = score;
+            c->fast_iter = iter;
+            c->fast_cs = cs;
+            c->fast_ncl = ncl;
+            c->fast_smem = smem;
+            c->fast_geom.NS = NS;
+            c->fast_geom.stash_off = NS * kCW * kCSlotBytes;
+            c->fast_geom.ncl = ncl;
+        }
     }
 }
 
-// The staged path needs bf16 rows of a multiple of 8 elements, long enough to give every
-// warp of a cluster work and short enough for the register stash.
-void staged_setup(adasd_ctx* c) {
-    c->staged_iter = 0;
-    c->staged_clusters[0] = c->staged_clusters[1] = 0;
-    const int V = c->cfg.V;
-    if (c->cfg.dtype != ADASD_BF16 || (V & 7) != 0 || V < 8192) return;
-    if (c->cfg.cluster_size != 0 && c->cfg.cluster_size != kSC) return;
-    const int NU = V >> 3;
-    const int per_cta = (NU + kSC - 1) / kSC;
-    const int per_warp = (per_cta + kSW - 1) / kSW + 1;
-    const int iter = (per_warp + 31) / 32;
-    if (iter > kStagedMaxIter) return;
-    c->staged_iter = iter;
-    c->staged_slice_pad = ((per_cta + 1) * 16 + 127) & ~127;
-    c->staged_clusters[0] = staged_prepare_iter<MODE_ADASD>(c);
-    c->staged_clusters[1] = staged_prepare_iter<MODE_VANILLA>(c);
-    if (c->staged_clusters[0] < 1 || c->staged_clusters[1] < 1) c->staged_iter = 0;
-}
-
 template <int ITER, int MODE>
-int staged_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
+int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
     const long long positions = (long long)p.B * (p.Kmax + 1);
-    int ncl = c->staged_clusters[MODE];
-    if (positions < ncl) ncl = (int)positions;
+    ClusterGeom gq = c->fast_geom;
+    if (positions < gq.ncl) gq.ncl = (int)positions;
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
-    lc.gridDim = dim3((unsigned)(ncl * kSC), 1, 1);
-    lc.blockDim = dim3(kSThreads, 1, 1);
-    lc.dynamicSmemBytes = 4 * c->staged_slice_pad;
+    lc.gridDim = dim3((unsigned)(gq.ncl * c->fast_cs), 1, 1);
+    lc.blockDim = dim3(kCThreads, 1, 1);
+    lc.dynamicSmemBytes = (size_t)c->fast_smem;
     lc.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kSC;
+    attr[0].val.clusterDim.x = (unsigned)c->fast_cs;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&lc, staged_verify_kernel<ITER, MODE>, p, ncl, c->staged_slice_pad));
+    CUDA_TRY(cudaLaunchKernelEx(&lc, cluster_verify_kernel<ITER, MODE>, p, gq));
     return ADASD_OK;
 }
 
 template <int MODE>
-int staged_launch_iter(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
-    switch (c->staged_iter) {
-        case 1: return staged_launch<1, MODE>(c, p, stream);
-        case 2: return staged_launch<2, MODE>(c, p, stream);
-        case 3: return staged_launch<3, MODE>(c, p, stream);
-        case 4: return staged_launch<4, MODE>(c, p, stream);
-        case 5: return staged_launch<5, MODE>(c, p, stream);
-        default: return ADASD_ERR_SHAPE;
-    }
+int fast_launch_iter(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
+#define CALL(I) fast_launch<I, MODE>(c, p, stream)
+    ADASD_ITER_SWITCH(c->fast_iter, CALL, ADASD_ERR_SHAPE)
+#undef CALL
 }
 
 int check_strides(const adasd_ctx* c, long long seq, long long row) {
@@ -218,7 +260,7 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
     const int cs = pick_cluster(ctx, positions);
     const bool vec = vec_ok(p.zd, ctx->cfg.dtype, {p.d_seq, p.d_row}) &&
                      vec_ok(p.zt, ctx->cfg.dtype, {p.t_seq, p.t_row});
-    if (vec && ctx->staged_iter > 0) return staged_launch_iter<MODE>(ctx, p, stream);
+    if (vec && ctx->fast_iter > 0) return fast_launch_iter<MODE>(ctx, p, stream);
     if (ctx->cfg.dtype == ADASD_BF16) {
         return vec ? launch_cluster(verify_kernel<__nv_bfloat16, true, MODE>, p, positions, cs, stream)
                    : launch_cluster(verify_kernel<__nv_bfloat16, false, MODE>, p, positions, cs, stream);
@@ -300,9 +342,7 @@ int adasd_create(adasd_ctx** out, const adasd_config* cfg) {
     if (cfg->kde_bandwidth < 0 || cfg->kde_bandwidth > 1 || cfg->reject_rule < 0 ||
         cfg->reject_rule > 1)
         return ADASD_ERR_DTYPE;
-    if (cfg->cluster_size != 0 && cfg->cluster_size != 1 && cfg->cluster_size != 2 &&
-        cfg->cluster_size != 4 && cfg->cluster_size != 8)
-        return ADASD_ERR_SHAPE;
+    if (cfg->cluster_size < 0 || cfg->cluster_size > kMaxCluster) return ADASD_ERR_SHAPE;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev)
         return ADASD_ERR_CUDA;
@@ -354,7 +394,7 @@ int adasd_create(adasd_ctx** out, const adasd_config* cfg) {
     ALLOC(t.van_tok, B * (K + 1));
     ALLOC(t.ticket, B);
 #undef ALLOC
-    if (rc == ADASD_OK) staged_setup(c);
+    if (rc == ADASD_OK) fast_setup(c, prop.sharedMemPerBlockOptin);
     if (rc == ADASD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ADASD_ERR_CUDA;
     if (rc != ADASD_OK) {
         for (void* q : c->allocs) cudaFree(q);

@@ -43,7 +43,7 @@ def test_strerror_and_null_arguments():
 def test_create_validates_before_touching_cuda():
     for field, value, want in (("B", 0, -3), ("V", 0, -3), ("Kmax", 0, -3), ("Kmax", 33, -3),
                                ("list_capacity", 0, -3), ("dtype", 7, -4), ("kde_bandwidth", 2, -4),
-                               ("reject_rule", -1, -4), ("cluster_size", 3, -3)):
+                               ("reject_rule", -1, -4), ("cluster_size", 9, -3)):
         cfg = adasd.AdasdConfig(4, 1000, 8, adasd.ADASD_BF16, 64, 0, 0, 2, 0, 0)
         setattr(cfg, field, value)
         rc, h = adasd.adasd_create(cfg)
