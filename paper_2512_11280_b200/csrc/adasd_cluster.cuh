@@ -32,6 +32,8 @@ constexpr int kCW = 12;                         // warps per CTA
 constexpr int kCThreads = kCW * 32;
 constexpr int kCMaxCluster = 8;
 constexpr int kCMaxG = kCMaxCluster * kCW;      // warps per cluster, at most
+constexpr int kCTab = 128;                      // entries of the per-warp tables (4 per lane)
+static_assert(kCMaxG <= kCTab, "per-warp tables hold one entry per warp of the cluster");
 constexpr int kCMaxSlots = 16;                  // ring slots per warp, at most
 constexpr int kCSlotBytes = 2048;               // 2 iterations x (512 B target + 512 B draft)
 constexpr int kCMaxIter = 10;                   // iterations per warp and row, at most
@@ -136,8 +138,8 @@ struct __align__(16) RowPart {
 struct __align__(16) ClusterShared {
     RowPart wtab[2][kCW];             // this CTA's warps, by position parity
     RowPart ctab[2][kCMaxCluster];    // every CTA's totals (written over DSMEM), by parity
-    float2 tabC[2][kCMaxG];           // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q)
-    float rtab[kCMaxG];               // vanilla: per-warp residual mass, every CTA holds all
+    float2 tabC[2][kCTab];            // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q)
+    float rtab[kCTab];                // vanilla: per-warp residual mass, every CTA holds all
     float fin[2][12];                 // leader: row totals kept for finalisation
     int32_t token[2];                 // leader: sampled token of the position
     int32_t tail_seq[2];              // leader: sequence whose tail must run (-1: none)
@@ -188,8 +190,8 @@ cluster_verify_kernel(VerifyParams p, ClusterGeom gq) {
         return reinterpret_cast<float4*>(stash + (size_t)(k - KR) * (kCW * kCSlotBytes) + plane * 512);
     };
 
-    if (threadIdx.x < 2 * kCMaxG) reinterpret_cast<float*>(sh.tabC)[threadIdx.x] = 0.f, reinterpret_cast<float*>(sh.tabC)[threadIdx.x + 2 * kCMaxG] = 0.f;
-    if (threadIdx.x < kCMaxG) sh.rtab[threadIdx.x] = 0.f;
+    for (int q = threadIdx.x; q < 4 * kCTab; q += kCThreads) reinterpret_cast<float*>(sh.tabC)[q] = 0.f;
+    if (threadIdx.x < kCTab) sh.rtab[threadIdx.x] = 0.f;
     if (threadIdx.x == 0) {
         sh.tail_seq[0] = sh.tail_seq[1] = -1;
         sh.cnt[0] = sh.cnt[1] = 0u;

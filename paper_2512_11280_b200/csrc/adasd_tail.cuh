@@ -75,7 +75,8 @@ __device__ __forceinline__ void kde_sums(const float* __restrict__ list, int n, 
         __syncthreads();
         if (threadIdx.x < 8 && i0 + threadIdx.x < K_t) {
             float a = 0.f;
-            for (int w = 0; w < kWarps; ++w) a += sh.red[w][threadIdx.x];
+            const int nw = (int)(blockDim.x >> 5);     // the CTA running the tail may have fewer warps
+            for (int w = 0; w < nw; ++w) a += sh.red[w][threadIdx.x];
             S[i0 + threadIdx.x] = a;
         }
     }
