@@ -266,7 +266,7 @@ def run_ours(args) -> dict:
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = oracle_sample(wl, args.cpu_seqs)
+        out["cpu_baseline"] = oracle_sample(synth.WORKLOADS[args.workload], args.cpu_seconds)
     if dist is not None:
         dist.destroy_process_group()
     return out if rank == 0 else None
@@ -274,29 +274,37 @@ def run_ours(args) -> dict:
 
 # ------------------------------------------------------------------------------ oracle arm
 
-def oracle_sample(wl, n_seq: int) -> dict:
-    """The oracle, as it stands, on n_seq sequences of one round of the workload: K draft
-    steps, the AdaSD verify round and the vanilla round.  Returns rows/s on the host cores."""
+def oracle_sample(wl, seconds: float, max_rounds: int = 4) -> dict:
+    """The oracle, as it stands, on whole rounds of the workload (every sequence: K draft
+    steps, the AdaSD verify round and the vanilla round) until about `seconds` of CPU work
+    are done.  Input generation is not timed.  Returns rows/s on the host cores."""
     import oracle
     cores = len(os.sched_getaffinity(0))
     K = wl.K
-    bl = np.arange(min(n_seq, wl.B), dtype=np.int32)
-    hd, ht = synth.host_round(wl, 0, bl)
-    U = synth.round_uniforms_cpu(wl, 0)
-    ud, ut, ua = U["draft"], U["target"], U["accept"]
     oracle.lib()
-    t0 = time.perf_counter()
-    rows = 0
-    for n, b in enumerate(bl):
-        st = oracle.SequenceState(capacity=1024)
-        x = [oracle.draft_step(hd[n, k], float(ud[b, k]), 0.0)["token"] for k in range(K)]
-        oracle.verify_round(st, hd[n], ht[n], x, ut[b], ua[b])
-        oracle.vanilla_round(hd[n], ht[n], x, U["vanilla_accept"][b], float(U["resample"][b]))
-        rows += K + 2 * (2 * K + 1)
-    dt = time.perf_counter() - t0
+    rows, dt, nseq, rounds = 0, 0.0, 0, 0
+    chunk = 16                                     # sequences generated and timed at a time
+    states = [oracle.SequenceState(capacity=4096) for _ in range(wl.B)]
+    while dt < seconds and rounds < max_rounds:
+        U = synth.round_uniforms_cpu(wl, rounds)
+        ud, ut, ua = U["draft"], U["target"], U["accept"]
+        for b0 in range(0, wl.B, chunk):
+            bl = np.arange(b0, min(b0 + chunk, wl.B), dtype=np.int32)
+            hd, ht = synth.host_round(wl, rounds, bl)
+            t0 = time.perf_counter()
+            for n, b in enumerate(bl):
+                x = [oracle.draft_step(hd[n, k], float(ud[b, k]), 0.0)["token"] for k in range(K)]
+                oracle.verify_round(states[b], hd[n], ht[n], x, ut[b], ua[b])
+                oracle.vanilla_round(hd[n], ht[n], x, U["vanilla_accept"][b], float(U["resample"][b]))
+                rows += K + 2 * (2 * K + 1)
+            dt += time.perf_counter() - t0
+            nseq += len(bl)
+            if dt >= seconds:
+                break
+        rounds += 1
     return {"value": rows / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{len(bl)} sequence(s) x 1 round of the workload ({rows} rows, {dt:.1f} s); "
-                      f"OpenMP over positions inside the verify round",
+            "sample": f"{nseq} sequence-rounds of the workload ({rows} rows, {dt:.1f} s of oracle time, "
+                      f"input generation excluded); OpenMP over positions inside the verify round",
             "seconds": dt}
 
 
@@ -309,12 +317,11 @@ def run_reference(args) -> dict:
     K = wl.K
     rows = step_rows(wl)
     for _ in range(min(args.warmup, 1)):
-        oracle_sample(wl, 1)
-    t0 = time.perf_counter()
+        oracle_sample(wl, 0.5, 1)
     total_rows, secs = 0, 0.0
     steps = max(1, min(args.steps, 6))
     for _ in range(steps):
-        s = oracle_sample(wl, 1)
+        s = oracle_sample(wl, 4.0, 1)
         total_rows += s["value"] * s["seconds"]
         secs += s["seconds"]
     value = total_rows / secs
@@ -324,10 +331,10 @@ def run_reference(args) -> dict:
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic",
             "config": {"workload": f"{args.workload}: B={wl.B} K={K} V={wl.V}; each step is a bounded "
-                                   f"sample: 1 sequence x 1 round ({K + 2 * (2 * K + 1)} rows of the "
-                                   f"{sum(rows.values())} a full step reads)"},
+                                   f"sample: about 4 s of oracle time on sequences of round 0 "
+                                   f"({K + 2 * (2 * K + 1)} rows per sequence of the {sum(rows.values())} a full step reads)"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": "1 sequence x 1 round per step"},
+                             "sample": "about 4 s of oracle time per step, sequences of round 0"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
 
@@ -341,7 +348,7 @@ def main():
     ap.add_argument("--workload", default="C4", choices=["C3", "C4"])
     ap.add_argument("--sets", type=int, default=4, help="input sets resident in HBM")
     ap.add_argument("--e2e-steps", type=int, default=6)
-    ap.add_argument("--cpu-seqs", type=int, default=2, help="sequences in the oracle sample")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="oracle time in the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
