@@ -12,6 +12,7 @@
 
 #include "adasd_rows.cuh"
 #include "adasd_cluster.cuh"
+#include "adasd_spec.cuh"
 
 using namespace adasd;
 
@@ -21,12 +22,14 @@ struct adasd_ctx {
     Scratch sc;
     std::vector<void*> allocs;
     int sm_count;
-    // streaming cluster kernel: fast_iter == 0 means not usable for this V / dtype
-    int fast_iter;            // iterations per warp and row (template parameter)
-    int fast_cs;              // CTAs per cluster
-    int fast_ncl;             // clusters resident at once (both modes)
-    int fast_smem;            // dynamic shared memory per CTA
-    ClusterGeom fast_geom;
+    // cluster kernels, one configuration per mode (AdaSD: warp-specialised kernel, vanilla:
+    // streaming cluster kernel); iter == 0 means not usable for this V / dtype
+    struct Fast {
+        int iter;             // iterations per warp and row (template parameter)
+        int cs;               // CTAs per cluster
+        int smem;             // dynamic shared memory per CTA
+        ClusterGeom geom;
+    } fast[2];
 };
 
 namespace {
@@ -88,9 +91,8 @@ int launch_cluster(void (*kernel)(P), const P& params, long long clusters, int c
 }
 
 // ---- streaming cluster kernel: configuration and launch ---------------------------------
-template <int ITER, int MODE>
-int fast_occupancy(int cs, int smem) {
-    auto kern = cluster_verify_kernel<ITER, MODE>;
+template <typename K>
+int kernel_occupancy(K kern, int threads, int cs, int smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
@@ -98,7 +100,7 @@ int fast_occupancy(int cs, int smem) {
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
     lc.gridDim = dim3((unsigned)(cs * 64), 1, 1);
-    lc.blockDim = dim3(kCThreads, 1, 1);
+    lc.blockDim = dim3((unsigned)threads, 1, 1);
     lc.dynamicSmemBytes = (size_t)smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -115,14 +117,26 @@ int fast_occupancy(int cs, int smem) {
     return n;
 }
 
-template <int ITER, int MODE>
-int fast_static_smem() {
+template <typename K>
+int kernel_static_smem(K kern) {
     cudaFuncAttributes fa;
-    if (cudaFuncGetAttributes(&fa, cluster_verify_kernel<ITER, MODE>) != cudaSuccess) {
+    if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) {
         cudaGetLastError();
         return -1;
     }
     return (int)fa.sharedSizeBytes;
+}
+
+// AdaSD mode runs the warp-specialised kernel, vanilla mode the streaming cluster kernel.
+template <int ITER, int MODE>
+int fast_occupancy(int cs, int smem) {
+    if (MODE == MODE_ADASD) return kernel_occupancy(spec_verify_kernel<ITER>, kSThreads, cs, smem);
+    return kernel_occupancy(cluster_verify_kernel<ITER, MODE_VANILLA>, kCThreads, cs, smem);
+}
+template <int ITER, int MODE>
+int fast_static_smem() {
+    if (MODE == MODE_ADASD) return kernel_static_smem(spec_verify_kernel<ITER>);
+    return kernel_static_smem(cluster_verify_kernel<ITER, MODE_VANILLA>);
 }
 
 #define ADASD_ITER_SWITCH(iter, CALL, fail)  \
@@ -140,83 +154,97 @@ int fast_static_smem() {
         default: return fail;                \
     }
 
+template <int MODE>
 int fast_occupancy_iter(int iter, int cs, int smem) {
-#define CALL(I) std::min(fast_occupancy<I, MODE_ADASD>(cs, smem), fast_occupancy<I, MODE_VANILLA>(cs, smem))
+#define CALL(I) fast_occupancy<I, MODE>(cs, smem)
     ADASD_ITER_SWITCH(iter, CALL, 0)
 #undef CALL
 }
+template <int MODE>
 int fast_static_smem_iter(int iter) {
-#define CALL(I) std::max(fast_static_smem<I, MODE_ADASD>(), fast_static_smem<I, MODE_VANILLA>())
+#define CALL(I) fast_static_smem<I, MODE>()
     ADASD_ITER_SWITCH(iter, CALL, -1)
 #undef CALL
 }
 
-// Chooses the cluster size that covers the most SMs among those whose per-CTA slice fits on
-// chip: the kept 2^t values (registers first, shared memory for the rest) plus a ring of at
-// least one position.  bf16 rows of a multiple of 8 elements only.
-void fast_setup(adasd_ctx* c, size_t smem_optin) {
-    c->fast_iter = 0;
+// Chooses, for one mode, the cluster size that covers the most SMs among those whose per-CTA
+// slice fits on chip: the kept 2^t values (registers first, shared memory for the rest) plus
+// a ring of at least one position.  bf16 rows of a multiple of 8 elements only.
+template <int MODE>
+void fast_setup_mode(adasd_ctx* c, size_t smem_optin) {
+    adasd_ctx::Fast& f = c->fast[MODE];
+    f.iter = 0;
     const int V = c->cfg.V;
     if (c->cfg.dtype != ADASD_BF16 || (V & 7) != 0 || V < 8192) return;
+    const int warps = (MODE == MODE_ADASD) ? kSW : kCW;          // warps that split a CTA's slice
+    const int reg_iter = (MODE == MODE_ADASD) ? kSRegIter : kCRegIter;
     const int NU = V >> 3;
     int best_score = 0;
     for (int cs = kCMaxCluster; cs >= 1; --cs) {
         if (c->cfg.cluster_size != 0 && c->cfg.cluster_size != cs) continue;
         const int ncu = (NU + cs - 1) / cs, nwi = (ncu + 31) / 32;
-        const int I_lo = nwi / kCW, rem = nwi % kCW, iter = I_lo + (rem ? 1 : 0);
+        const int I_lo = nwi / warps, rem = nwi % warps, iter = I_lo + (rem ? 1 : 0);
         if (iter < 1 || iter > kCMaxIter) continue;
-        const int KR = std::min(iter, kCRegIter);
+        const int KR = std::min(iter, reg_iter);
         int stash_slots = 0;
-        if (iter > KR) stash_slots = (iter - 1 - KR) * kCW + ((iter - 1 < I_lo) ? kCW : rem);
+        if (iter > KR) stash_slots = (iter - 1 - KR) * warps + ((iter - 1 < I_lo) ? warps : rem);
         const int stash_bytes = stash_slots * kCSlotBytes;
-        const int st = fast_static_smem_iter(iter);
+        const int st = fast_static_smem_iter<MODE>(iter);
         if (st < 0) continue;
         const int avail = (int)smem_optin - st - stash_bytes - 1024;
         const int n_stg = (iter + 1) / 2;
-        int NS = std::min({kCMaxSlots, avail / (kCW * kCSlotBytes), 2 * n_stg});
+        int NS = std::min({kCMaxSlots, avail / (warps * kCSlotBytes), 2 * n_stg});
         if (NS < n_stg) continue;
-        const int smem = NS * kCW * kCSlotBytes + stash_bytes;
-        const int ncl = fast_occupancy_iter(iter, cs, smem);
+        const int smem = NS * warps * kCSlotBytes + stash_bytes;
+        const int ncl = fast_occupancy_iter<MODE>(iter, cs, smem);
         const int score = ncl * cs;
         if (score > best_score) {
             best_score = score;
-            c->fast_iter = iter;
-            c->fast_cs = cs;
-            c->fast_ncl = ncl;
-            c->fast_smem = smem;
-            c->fast_geom.NS = NS;
-            c->fast_geom.stash_off = NS * kCW * kCSlotBytes;
-            c->fast_geom.ncl = ncl;
+            f.iter = iter;
+            f.cs = cs;
+            f.smem = smem;
+            f.geom.NS = NS;
+            f.geom.stash_off = NS * warps * kCSlotBytes;
+            f.geom.ncl = ncl;
         }
     }
+}
+void fast_setup(adasd_ctx* c, size_t smem_optin) {
+    fast_setup_mode<MODE_ADASD>(c, smem_optin);
+    fast_setup_mode<MODE_VANILLA>(c, smem_optin);
 }
 
 template <int ITER, int MODE>
 int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
     const long long positions = (long long)p.B * (p.Kmax + 1);
-    ClusterGeom gq = c->fast_geom;
+    const adasd_ctx::Fast& f = c->fast[MODE];
+    ClusterGeom gq = f.geom;
     if (positions < gq.ncl) gq.ncl = (int)positions;
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
-    lc.gridDim = dim3((unsigned)(gq.ncl * c->fast_cs), 1, 1);
-    lc.blockDim = dim3(kCThreads, 1, 1);
-    lc.dynamicSmemBytes = (size_t)c->fast_smem;
+    lc.gridDim = dim3((unsigned)(gq.ncl * f.cs), 1, 1);
+    lc.blockDim = dim3((unsigned)(MODE == MODE_ADASD ? kSThreads : kCThreads), 1, 1);
+    lc.dynamicSmemBytes = (size_t)f.smem;
     lc.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)c->fast_cs;
+    attr[0].val.clusterDim.x = (unsigned)f.cs;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&lc, cluster_verify_kernel<ITER, MODE>, p, gq));
+    if (MODE == MODE_ADASD) {
+        CUDA_TRY(cudaLaunchKernelEx(&lc, spec_verify_kernel<ITER>, p, gq));
+    } else {
+        CUDA_TRY(cudaLaunchKernelEx(&lc, cluster_verify_kernel<ITER, MODE_VANILLA>, p, gq));
+    }
     return ADASD_OK;
 }
 
 template <int MODE>
 int fast_launch_iter(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
 #define CALL(I) fast_launch<I, MODE>(c, p, stream)
-    ADASD_ITER_SWITCH(c->fast_iter, CALL, ADASD_ERR_SHAPE)
+    ADASD_ITER_SWITCH(c->fast[MODE].iter, CALL, ADASD_ERR_SHAPE)
 #undef CALL
 }
 
@@ -260,7 +288,7 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
     const int cs = pick_cluster(ctx, positions);
     const bool vec = vec_ok(p.zd, ctx->cfg.dtype, {p.d_seq, p.d_row}) &&
                      vec_ok(p.zt, ctx->cfg.dtype, {p.t_seq, p.t_row});
-    if (vec && ctx->fast_iter > 0) return fast_launch_iter<MODE>(ctx, p, stream);
+    if (vec && ctx->fast[MODE].iter > 0) return fast_launch_iter<MODE>(ctx, p, stream);
     if (ctx->cfg.dtype == ADASD_BF16) {
         return vec ? launch_cluster(verify_kernel<__nv_bfloat16, true, MODE>, p, positions, cs, stream)
                    : launch_cluster(verify_kernel<__nv_bfloat16, false, MODE>, p, positions, cs, stream);

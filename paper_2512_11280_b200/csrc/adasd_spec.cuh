@@ -1,0 +1,974 @@
+// Warp-specialised AdaSD verification kernel for sm_100a.
+//
+// Same data path as the streaming cluster kernel (persistent clusters, per-warp slot rings
+// filled by 1-D bulk copies, 2^t values kept in registers and shared memory, every logit row
+// read from HBM once), but the irregular work is taken off the arithmetic warps:
+//
+//  * 10 COMPUTE warps per CTA do nothing but the three passes over their share of a position
+//    (maxima; 2^t, S and T; (p+q) log2 (p+q)), the refill of their own ring slots and, for
+//    the one warp that holds it, the inverse-CDF crossing.
+//  * 1 CONTROL warp per CTA finds the cluster's positions, folds the warp partials into the
+//    CTA's totals, exchanges them with the other CTAs of the cluster (DSMEM stores + remote
+//    mbarrier arrivals: no cluster-wide barrier in the loop), turns the row totals into one
+//    small message per compute warp (its scale factors and whether it holds the crossing) and,
+//    in the leader CTA, finalises the previous position and draws the sequence's ticket.
+//  * 1 TAIL warp per CTA runs the tails (KDE/Bayes, accept scan, list appends, T_G) of the
+//    sequences its control warp completes, off everybody's critical path.
+//
+// Every wait (slot filled, partials in, totals in, message ready, sums in, queue) is bounded:
+// a warp whose wait expires sets ADASD_STATUS_TIMEOUT, stops waiting and copying, and walks
+// through the rest of the protocol, so the kernel always ends.
+#pragma once
+
+#include "adasd_cluster.cuh"
+
+namespace adasd {
+
+constexpr int kSW = 10;                          // compute warps per CTA
+constexpr int kSCtl = kSW;                       // warp index of the control warp
+constexpr int kSTail = kSW + 1;                  // warp index of the tail warp
+constexpr int kSThreads = (kSW + 2) * 32;        // 384: leaves 168 registers per thread
+constexpr int kSRegIter = 6;                     // iterations whose 2^t values stay in registers
+static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
+constexpr int kSPosRing = 8;                     // positions the control warp keeps described
+constexpr int kSQueue = 64;                      // tail queue entries
+constexpr uint32_t kSPollSpins = 1u << 24;       // polls of the tail queue before giving up
+
+// One position as the control warp describes it to the compute warps of its CTA.
+struct __align__(16) PosCtx {
+    unsigned long long src_t;     // global address of the CTA's slice of the target row
+    unsigned long long src_d;     // ... of the draft row (unused for a bonus row)
+    int32_t pos;                  // index into [B, Kmax+1]; >= total: none
+    int32_t kt;                   // window K_t of its sequence
+    int32_t bonus;                // 1: the sequence's bonus row (target row only)
+    int32_t pad;
+};
+
+// What a compute warp needs after the exchange: p = 2^t_p * at, q = 2^t_q * ad; and, if it
+// holds the inverse-CDF crossing (sel), the weight before its share and the target.
+struct __align__(16) WarpMsg {
+    float at, ad, ft, base;
+    float target;
+    int32_t sel;
+    int32_t pad0, pad1;
+};
+
+struct __align__(16) SpecShared {
+    PosCtx pc[kSPosRing];
+    RowPart wtab[2][kCW];             // this CTA's compute warps, by position parity
+    RowPart ctab[2][kCMaxCluster];    // every CTA's totals (written over DSMEM), by parity
+    WarpMsg wmsg[2][kCW];
+    float2 tabC[2][kCTab];            // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q)
+    float fin[2][8];                  // leader: row totals kept for finalisation
+    int32_t token[2];                 // leader: sampled token of the position
+    unsigned long long entry_bar[2];  // one arrival per compute warp: wtab[par] complete
+    unsigned long long ctab_bar[2];   // CS remote arrivals: ctab[par] complete
+    unsigned long long scal_bar[2];   // 1 arrival: wmsg[par] ready
+    unsigned long long c_bar[2];      // leader: one remote arrival per compute warp of the cluster: tabC[par], token[par] complete
+    unsigned long long bar[kCW][kCMaxSlots];   // "slot filled" barriers
+    int32_t tq[kSQueue];              // leader: sequences whose tail must run (-1: stop)
+    uint32_t tq_head, tq_tail;        // pushed by the control warp / done by the tail warp
+    float td[ADASD_KMAX_LIMIT], tH[ADASD_KMAX_LIMIT];   // tail warp scratch
+};
+
+// ---- mbarrier helpers with explicit scopes -----------------------------------------------
+__device__ __forceinline__ void mbar_arrive_cta(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// arrival on the same barrier in CTA `cta` of the cluster; releases this thread's earlier
+// writes (its DSMEM stores included) to whoever acquires at cluster scope
+__device__ __forceinline__ void mbar_arrive_remote(uint64_t* bar, uint32_t cta) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(smem_u32(bar)), "r"(cta)
+        : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kCWaitSpins; ++it)
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+    return false;
+}
+
+// The per-sequence tail of a round, run by ONE warp: lane i owns candidate i.  Same
+// arithmetic as verify_tail (KDE sums over L_D^A and L_D^R, Bayes posterior with the
+// round's earlier distances counted as accepted, first-rejection scan, appends, T_G).
+// sd/sH: 32-entry shared-memory scratch of this warp.
+__device__ __forceinline__ void verify_tail_warp(const TailConfig& cfg, const TailIO& io, State& st, int b,
+                                                 float* sd, float* sH) {
+    const int lane = threadIdx.x & 31;
+    const int Kmax = cfg.Kmax;
+    int K_t = io.draft_len ? __ldcg(io.draft_len + b) : Kmax;
+    K_t = max(0, min(K_t, Kmax));
+    float d = 0.f, H = 0.f, u = 0.f;
+    int x = 0, y = 0;
+    if (lane < K_t) {
+        d = __ldcg(io.dist + (size_t)b * Kmax + lane);
+        H = __ldcg(io.H_d + (size_t)b * Kmax + lane);
+        y = __ldcg(io.y + (size_t)b * (Kmax + 1) + lane);
+        x = io.x[(size_t)b * Kmax + lane];
+        u = io.u_accept[(size_t)b * Kmax + lane];
+        sd[lane] = d;
+        sH[lane] = H;
+    }
+    __syncwarp();
+    const int nA0 = st.nA[b], nR0 = st.nR[b];
+    const bool inside = d > 0.f && d < 1.f;          // enters the KDE lists when accepted
+
+    // bandwidths: candidate i sees L_D^A plus the distances d_1..d_{i-1} of this round that
+    // lie strictly inside (0,1): the list "as it stands" when candidate i is reached at all
+    double n = (double)nA0, s = st.sumA[b], s2 = st.sumA2[b];
+    for (int j = 0; j < K_t; ++j) {
+        const float dj = __shfl_sync(0xFFFFFFFFu, d, j);
+        if (j < lane && dj > 0.f && dj < 1.f) {
+            n += 1.0;
+            s += (double)dj;
+            s2 += (double)dj * (double)dj;
+        }
+    }
+    const double hA = kde_bandwidth(n, s, s2, cfg.bw_rule);
+    const bool ok = lane < K_t && (n >= (double)cfg.min_samples) && (hA > 0.0);
+    const float cA = ok ? (float)(-0.5 * 1.4426950408889634 / (hA * hA)) : 0.f;
+    const float ihA = ok ? (float)(1.0 / hA) : 0.f;
+    const double hR = kde_bandwidth((double)nR0, st.sumR[b], st.sumR2[b], cfg.bw_rule);
+    const bool validR = (nR0 >= cfg.min_samples) && (hR > 0.0);
+    const float cR = validR ? (float)(-0.5 * 1.4426950408889634 / (hR * hR)) : 0.f;
+    const float ihR = validR ? (float)(1.0 / hR) : 0.f;
+    const bool any_valid = (__ballot_sync(0xFFFFFFFFu, ok) != 0u) && validR;
+
+    float SA = 0.f, SR = 0.f;
+    if (any_valid) {
+        const float* LA = st.LA + (size_t)b * st.cap;
+        const float* LR = st.LR + (size_t)b * st.cap;
+        for (int i0 = 0; i0 < K_t; i0 += 8) {
+            float accA[8], accR[8], di[8], ci[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int i = min(i0 + k, K_t - 1);
+                accA[k] = accR[k] = 0.f;
+                di[k] = __shfl_sync(0xFFFFFFFFu, d, i);
+                ci[k] = __shfl_sync(0xFFFFFFFFu, cA, i);
+            }
+            for (int j = lane; j < nA0; j += 32) {
+                const float xj = __ldcg(LA + j);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float t = di[k] - xj;
+                    accA[k] += ex2(ci[k] * t * t);
+                }
+            }
+            for (int j = lane; j < nR0; j += 32) {
+                const float xj = __ldcg(LR + j);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float t = di[k] - xj;
+                    accR[k] += ex2(cR * t * t);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float a = warp_sum(accA[k]), r = warp_sum(accR[k]);
+                if (lane == i0 + k) {
+                    SA = a;
+                    SR = r;
+                }
+            }
+        }
+    }
+    // kernel terms of this round's earlier distances, then the posterior
+    float extra = 0.f;
+    for (int j = 0; j < K_t; ++j) {
+        const float dj = __shfl_sync(0xFFFFFFFFu, d, j);
+        if (j < lane && dj > 0.f && dj < 1.f) {
+            const float t = d - dj;
+            extra += ex2(cA * t * t);
+        }
+    }
+    float P = 0.f;
+    if (any_valid && ok) {
+        // n_A f_A = SA / (h_A sqrt(2 pi)),  n_R f_R = SR / (h_R sqrt(2 pi))
+        const float a = (SA + extra) * ihA;
+        const float r = SR * ihR;
+        const float den = a + r;
+        if (den > 0.f && den < INFINITY) P = a / den;
+    }
+    if (lane < K_t) {
+        io.p_acc[(size_t)b * Kmax + lane] = P;
+        if (io.p_acc_user) io.p_acc_user[(size_t)b * Kmax + lane] = P;
+    }
+    const bool rej = cfg.reject_rule == 0 ? (u >= P) : (P < 0.5f);
+    const unsigned m = __ballot_sync(0xFFFFFFFFu, lane < K_t && x != y && rej);
+    (void)inside;
+    if (lane == 0) {
+        const int w = m ? (__ffs(m) - 1) : K_t;
+        const bool rejected = (m != 0u);
+        io.accept_len[b] = w;
+        io.next_token[b] = __ldcg(io.y + (size_t)b * (Kmax + 1) + w);
+        if (io.accept_len_rec) io.accept_len_rec[b] = w;
+        if (io.rejected_rec) io.rejected_rec[b] = rejected ? 1 : 0;
+        if (io.draft_len_rec) io.draft_len_rec[b] = K_t;
+        if (cfg.update) apply_update(st, b, w, rejected, sd, sH);
+    }
+    __syncwarp();
+}
+
+// ------------------------------------------------------------------------------------
+template <int ITER>
+__global__ void __launch_bounds__(kSThreads, 1)
+spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
+    constexpr int KR = ITER < kSRegIter ? ITER : kSRegIter;   // iterations kept in registers
+    constexpr int NSTG = (ITER + 1) / 2;                      // slots of one position, at most
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ SpecShared sh;
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int CS = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+    const int cid = blockIdx.x / CS;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int Kmax = p.Kmax, K1 = Kmax + 1;
+    const int total = p.B * K1;
+    const int ncl = gq.ncl;
+    const bool leader = (rank == 0);
+    const int NU = p.V >> 3;                                   // 16-byte units per row
+    const int cu0 = (int)((long long)rank * NU / CS), cu1 = (int)((long long)(rank + 1) * NU / CS);
+
+    for (int q = threadIdx.x; q < 4 * kCTab; q += kSThreads) reinterpret_cast<float*>(sh.tabC)[q] = 0.f;
+    if (threadIdx.x < kSPosRing) {
+        sh.pc[threadIdx.x].pos = total;
+        sh.pc[threadIdx.x].kt = 0;
+        sh.pc[threadIdx.x].bonus = 0;
+    }
+    if (threadIdx.x == 0) {
+        sh.token[0] = sh.token[1] = -1;
+        sh.tq_head = sh.tq_tail = 0u;
+        for (int k = 0; k < 2; ++k) {
+            mbar_init(reinterpret_cast<uint64_t*>(&sh.entry_bar[k]), kSW);
+            mbar_init(reinterpret_cast<uint64_t*>(&sh.ctab_bar[k]), (uint32_t)CS);
+            mbar_init(reinterpret_cast<uint64_t*>(&sh.scal_bar[k]), 1);
+            mbar_init(reinterpret_cast<uint64_t*>(&sh.c_bar[k]), (uint32_t)(CS * kSW));
+        }
+    }
+    if (warp < kSW && lane == 0)
+        for (int s = 0; s < kCMaxSlots; ++s) mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][s]), 1);
+    __syncthreads();
+
+    // first active position among start, start + ncl, ... (32 candidates per round)
+    auto window = [&](int b) -> int {
+        int kt = p.draft_len ? __ldg(p.draft_len + b) : Kmax;
+        return max(0, min(kt, Kmax));
+    };
+    auto scan_from = [&](int start) -> PosRef {
+        PosRef r;
+        r.pos = total;
+        r.kt = 0;
+        for (int base = start; base < total; base += 32 * ncl) {
+            const long long cl = (long long)base + (long long)lane * ncl;
+            int kt = 0;
+            bool ok = false;
+            if (cl < total) {
+                const int c = (int)cl, b = c / K1;
+                kt = window(b);
+                ok = (c - b * K1) <= kt;
+            }
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, ok);
+            if (m) {
+                const int src = __ffs(m) - 1;
+                r.pos = base + src * ncl;
+                r.kt = __shfl_sync(0xFFFFFFFFu, kt, src);
+                break;
+            }
+        }
+        return r;
+    };
+    // control warp: describe position number n to the compute warps
+    auto set_pos = [&](int n, const PosRef& r) {
+        if (lane == 0) {
+            PosCtx& c = sh.pc[n & (kSPosRing - 1)];
+            c.pos = r.pos;
+            c.kt = r.kt;
+            if (r.pos < total) {
+                const int b = r.pos / K1, i = r.pos - b * K1;
+                c.bonus = (i == r.kt) ? 1 : 0;
+                c.src_t = (unsigned long long)(reinterpret_cast<const __nv_bfloat16*>(p.zt) + (long long)b * p.t_seq +
+                                               (long long)i * p.t_row + (size_t)cu0 * 8);
+                c.src_d = (unsigned long long)(reinterpret_cast<const __nv_bfloat16*>(p.zd) + (long long)b * p.d_seq +
+                                               (long long)i * p.d_row + (size_t)cu0 * 8);
+            }
+        }
+        __syncwarp();
+    };
+    PosRef lastp;               // control warp: the latest position it has described
+    lastp.pos = total;
+    lastp.kt = 0;
+    if (warp == kSCtl) {
+        PosRef r = scan_from(cid);
+        set_pos(0, r);
+        for (int n = 1; n < 3; ++n) {
+            if (r.pos < total) r = scan_from(r.pos + ncl);
+            set_pos(n, r);
+        }
+        lastp = r;
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    cluster.sync();   // barriers and positions are set up in every CTA of the cluster
+
+    bool alive = true;         // false after a wait expired: this warp stops waiting and copying
+    auto expired = [&]() {
+        alive = false;
+        if (lane == 0) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+    };
+    auto wait_cta = [&](unsigned long long* bar, uint32_t par) {
+        if (!alive) return;
+        bool ok = mbar_wait_bounded(reinterpret_cast<uint64_t*>(bar), par);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) expired();
+    };
+    auto wait_cluster = [&](unsigned long long* bar, uint32_t par) {
+        if (!alive) return;
+        bool ok = mbar_wait_bounded_cluster(reinterpret_cast<uint64_t*>(bar), par);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) expired();
+    };
+
+    if (warp < kSW) {
+        // ============================== compute warp ======================================
+        // Its share of a row: iterations [wi0, wi0 + I_w) of the CTA's slice; the host sizes
+        // ITER so that every warp of every CTA gets ITER - 1 or ITER iterations.
+        const int g = rank * kSW + warp;
+        const int nwi = (cu1 - cu0 + 31) >> 5;                     // warp-iterations of this CTA
+        const int I_lo = nwi / kSW, I_rem = nwi % kSW;
+        const int I_w = min(ITER, I_lo + (warp < I_rem ? 1 : 0));
+        const bool full = (I_w == ITER);                           // the last iteration exists
+        const int wi0 = warp * I_lo + min(warp, I_rem);
+        const int wu0 = cu0 + 32 * wi0;
+        const int nwu = max(0, min(32 * I_w, cu1 - wu0));          // units of this warp (last one ragged)
+        const int n_stg = (I_w + 1) >> 1;                          // ring slots one position takes
+        const int NSw = min(gq.NS, 2 * n_stg);                     // slots this warp cycles through
+        const uint32_t last_bytes = n_stg > 0 ? (uint32_t)(nwu - 64 * (n_stg - 1)) * 16u : 0u;
+        const size_t woff = (size_t)wi0 * 512;                     // byte offset of the share in the CTA's slice
+
+        unsigned char* const ring = dyn_smem + (size_t)warp * gq.NS * kCSlotBytes;
+        unsigned char* const stash = dyn_smem + gq.stash_off + (size_t)warp * kCSlotBytes + (size_t)lane * 16;
+        auto stash_ptr = [&](int k, int plane) -> float4* {
+            return reinterpret_cast<float4*>(stash + (size_t)(k - KR) * (kSW * kCSlotBytes) + plane * 512);
+        };
+        auto pcx = [&](int n) -> const PosCtx& { return sh.pc[n & (kSPosRing - 1)]; };
+
+        int n = 0;                 // sequence number of the current position
+        uint32_t phase = 0;        // bit s: parity to wait for on slot s
+        int cons_slot = 0;         // slot holding the next stage to be consumed
+        int ip_which = 0;          // position the next fill belongs to: n + ip_which (at most n + 2)
+        int ip_stage = 0;          // its next stage
+        auto bar_of = [&](int s) -> uint64_t* { return reinterpret_cast<uint64_t*>(&sh.bar[warp][s]); };
+        auto issue_one = [&](int slot) {
+            if (!alive || n_stg == 0 || ip_which > 2) return;
+            const PosCtx& c = pcx(n + ip_which);
+            if (c.pos >= total) return;
+            if (lane == 0) {
+                const uint32_t bytes = (ip_stage == n_stg - 1) ? last_bytes : 1024u;
+                const bool bonus = c.bonus != 0;
+                unsigned char* dst = ring + (size_t)slot * kCSlotBytes;
+                uint64_t* bar = bar_of(slot);
+                const size_t off = woff + (size_t)ip_stage * 1024;
+                mbar_expect_tx(bar, bonus ? bytes : 2u * bytes);
+                bulk_g2s(dst, reinterpret_cast<const unsigned char*>(c.src_t) + off, bytes, bar);
+                if (!bonus) bulk_g2s(dst + 1024, reinterpret_cast<const unsigned char*>(c.src_d) + off, bytes, bar);
+            }
+            if (++ip_stage == n_stg) {
+                ip_stage = 0;
+                ++ip_which;
+            }
+        };
+        for (int s = 0; s < NSw; ++s) issue_one(s);
+
+        // iteration k runs for this warp: all but the last always do
+        auto k_on = [&](int k) -> bool { return (k < ITER - 1) || full; };
+        // Only one of a warp's last two iterations can be ragged (the CTA's slice need not end
+        // on a 32-unit boundary): lanes past the end take the clamp value, i.e. probability 0.
+        auto mask_unit = [&](int k, uint4& w) {
+            if (k >= ITER - 2 && !(lane + 32 * k < nwu))
+                w = make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
+        };
+
+        // ---- pass A: packed maxima and flags of one position, slot by slot ------------------
+        uint32_t a_mT = 0xFF80FF80u, a_mD = 0xFF80FF80u, a_df = 0u;   // -inf pairs
+        int a_next = 0;                                                 // first stage not yet scanned
+        auto pass_a = [&](auto bonus_c, bool blocking) {
+            constexpr bool BONUS = decltype(bonus_c)::value;
+            if (!alive) return;
+#pragma unroll
+            for (int st = 0; st < NSTG; ++st) {
+                if (st >= a_next && st < n_stg) {
+                    int slot = cons_slot + st;
+                    if (slot >= NSw) slot -= NSw;
+                    const uint32_t par = (phase >> slot) & 1u;
+                    bool ok = blocking ? mbar_wait_bounded(bar_of(slot), par)
+                                       : (mbar_test_wait(bar_of(slot), par) != 0);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) {
+                        if (blocking) expired();     // the copy never landed
+                        break;
+                    }
+                    a_next = st + 1;
+                    const unsigned char* sb = ring + (size_t)slot * kCSlotBytes + (size_t)lane * 16;
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) {
+                        const int k = 2 * st + kk;
+                        if (k < ITER && k_on(k)) {
+                            uint4 T = *reinterpret_cast<const uint4*>(sb + kk * 512);
+                            mask_unit(k, T);
+                            a_mT = bmax2(bmax2(a_mT, T.x), bmax2(T.y, bmax2(T.z, T.w)));
+                            if (!BONUS) {
+                                uint4 D = *reinterpret_cast<const uint4*>(sb + 1024 + kk * 512);
+                                mask_unit(k, D);
+                                a_mD = bmax2(bmax2(a_mD, D.x), bmax2(D.y, bmax2(D.z, D.w)));
+                                a_df |= (T.x ^ D.x) | (T.y ^ D.y) | (T.z ^ D.z) | (T.w ^ D.w);
+                            }
+                        }
+                    }
+                }
+            }
+        };
+        auto pass_a_any = [&](bool bonus, bool blocking) {
+            if (bonus) pass_a(std::true_type{}, blocking);
+            else pass_a(std::false_type{}, blocking);
+        };
+
+        // The warp's shifts and flags from the packed accumulators.  Shifts live in the log2
+        // domain: M = fl(max * log2 e), and every kept value is 2^(z log2 e - M) with ONE
+        // rounding (an FMA), so sums of different warps combine through the exact differences
+        // of their M.  A slice without a finite logit gets M = kFloorL and all-zero values.
+        float Mt_w = kFloorL, Md_w = kFloorL;
+        float nmt_w = 0.f, nmd_w = 0.f;           // FMA addends of pass B (-M, or 0 for an empty slice)
+        uint32_t flags_w = 0;
+        auto finish_a = [&](bool bonus) {
+            const float2 a = unpack2(a_mT), d = unpack2(a_mD);
+            uint32_t bad = (a.x != a.x || a.y != a.y || d.x != d.x || d.y != d.y) ? 1u : 0u;
+            const float vt = warp_max_f32(fmaxf(a.x, a.y));
+            const float vd = bonus ? vt : warp_max_f32(fmaxf(d.x, d.y));
+            if (vt == INFINITY || vd == INFINITY || !alive) bad = 1u;
+            const bool has_t = vt > ADASD_FLOOR_BF, has_d = vd > ADASD_FLOOR_BF;
+            Mt_w = has_t ? vt * kLog2e : kFloorL;
+            Md_w = has_d ? vd * kLog2e : kFloorL;
+            nmt_w = has_t ? -Mt_w : 0.f;
+            nmd_w = has_d ? -Md_w : 0.f;
+            flags_w = __reduce_or_sync(0xFFFFFFFFu, bad | (a_df ? 2u : 0u));
+            a_mT = a_mD = 0xFF80FF80u;
+            a_df = 0u;
+            a_next = 0;
+        };
+
+        // ---- pass B: 2^t values (kept) and the warp's S and T --------------------------------
+        float et[KR][8], ed[KR][8];
+        float sB[4];                       // after pass_b: warp totals St, Tt, Sd, Td
+        auto pass_b = [&](auto bonus_c) {
+            constexpr bool BONUS = decltype(bonus_c)::value;
+            float2 St = make_float2(0.f, 0.f), Tt = St, Sd = St, Td = St;
+            const float2 L2 = make_float2(kLog2e, kLog2e);
+            const float2 nmt = make_float2(nmt_w, nmt_w);
+            const float2 nmd = make_float2(nmd_w, nmd_w);
+#pragma unroll
+            for (int st = 0; st < NSTG; ++st) {
+                if ((2 * st < ITER - 1) || full) {                       // the stage exists for this warp
+                    const unsigned char* sb = ring + (size_t)cons_slot * kCSlotBytes + (size_t)lane * 16;
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) {
+                        const int k = 2 * st + kk;
+                        if (k < ITER && k_on(k)) {
+                            float e1[8], e2[8];
+                            uint4 T = *reinterpret_cast<const uint4*>(sb + kk * 512);
+                            mask_unit(k, T);
+                            const uint32_t tw[4] = {T.x, T.y, T.z, T.w};
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float2 z = unpack2(bclamp2(tw[j]));
+                                const float2 t = __ffma2_rn(z, L2, nmt);
+                                const float2 e = make_float2(ex2(t.x), ex2(t.y));
+                                e1[2 * j] = e.x;
+                                e1[2 * j + 1] = e.y;
+                                St = __fadd2_rn(St, e);
+                                Tt = __ffma2_rn(e, t, Tt);
+                            }
+                            if (!BONUS) {
+                                uint4 D = *reinterpret_cast<const uint4*>(sb + 1024 + kk * 512);
+                                mask_unit(k, D);
+                                const uint32_t dw[4] = {D.x, D.y, D.z, D.w};
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const float2 z = unpack2(bclamp2(dw[j]));
+                                    const float2 t = __ffma2_rn(z, L2, nmd);
+                                    const float2 e = make_float2(ex2(t.x), ex2(t.y));
+                                    e2[2 * j] = e.x;
+                                    e2[2 * j + 1] = e.y;
+                                    Sd = __fadd2_rn(Sd, e);
+                                    Td = __ffma2_rn(e, t, Td);
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) e2[j] = 0.f;
+                            }
+                            if (k < KR) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    et[k < KR ? k : 0][j] = e1[j];
+                                    ed[k < KR ? k : 0][j] = e2[j];
+                                }
+                            } else {
+                                *stash_ptr(k, 0) = make_float4(e1[0], e1[1], e1[2], e1[3]);
+                                *stash_ptr(k, 1) = make_float4(e1[4], e1[5], e1[6], e1[7]);
+                                if (!BONUS) {
+                                    *stash_ptr(k, 2) = make_float4(e2[0], e2[1], e2[2], e2[3]);
+                                    *stash_ptr(k, 3) = make_float4(e2[4], e2[5], e2[6], e2[7]);
+                                }
+                            }
+                        }
+                    }
+                    // the slot is consumed: flip its parity and refill it with the next stage
+                    __syncwarp();
+                    phase ^= 1u << cons_slot;
+                    issue_one(cons_slot);
+                    if (++cons_slot == NSw) cons_slot = 0;
+                }
+            }
+            sB[0] = warp_sum(St.x + St.y);
+            sB[1] = warp_sum(Tt.x + Tt.y);
+            if (BONUS) {
+                sB[2] = sB[0];
+                sB[3] = sB[1];
+            } else {
+                sB[2] = warp_sum(Sd.x + Sd.y);
+                sB[3] = warp_sum(Td.x + Td.y);
+            }
+        };
+        // the 2^t values of iteration k (compile-time k after unrolling)
+        auto load_stash = [&](int k, float (&a)[8], float (&b)[8]) {
+            if (k < KR) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    a[j] = et[k < KR ? k : 0][j];
+                    b[j] = ed[k < KR ? k : 0][j];
+                }
+            } else {
+                const float4 a0 = *stash_ptr(k, 0), a1 = *stash_ptr(k, 1), b0 = *stash_ptr(k, 2), b1 = *stash_ptr(k, 3);
+                a[0] = a0.x, a[1] = a0.y, a[2] = a0.z, a[3] = a0.w, a[4] = a1.x, a[5] = a1.y, a[6] = a1.z, a[7] = a1.w;
+                b[0] = b0.x, b[1] = b0.y, b[2] = b0.z, b[3] = b0.w, b[4] = b1.x, b[5] = b1.y, b[6] = b1.z, b[7] = b1.w;
+            }
+        };
+        auto load_stash_t = [&](int k, float (&a)[8]) {      // target values only
+            if (k < KR) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) a[j] = et[k < KR ? k : 0][j];
+            } else {
+                const float4 a0 = *stash_ptr(k, 0), a1 = *stash_ptr(k, 1);
+                a[0] = a0.x, a[1] = a0.y, a[2] = a0.z, a[3] = a0.w, a[4] = a1.x, a[5] = a1.y, a[6] = a1.z, a[7] = a1.w;
+            }
+        };
+
+        // Run by the warp that holds the crossing: first element (index order: iteration, lane,
+        // element) of the target row where base + f * running weight exceeds target, else the
+        // last element with weight.
+        auto select_kept = [&](float base, float f, float target) -> int {
+            float ls[ITER], tot[ITER];
+#pragma unroll
+            for (int k = 0; k < ITER; ++k) {
+                ls[k] = 0.f;
+                if (k_on(k)) {
+                    float v[8];
+                    load_stash_t(k, v);
+                    ls[k] = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < ITER; ++k) tot[k] = warp_sum(ls[k]);
+            int ksel = -1, klast = -1;
+            float run = 0.f, runsel = 0.f, runlast = 0.f;
+#pragma unroll
+            for (int k = 0; k < ITER; ++k) {
+                if (tot[k] > 0.f) {
+                    klast = k;
+                    runlast = run;
+                    if (ksel < 0 && fmaf(f, run + tot[k], base) > target) {
+                        ksel = k;
+                        runsel = run;
+                    }
+                }
+                run += tot[k];
+            }
+            if (ksel < 0) {
+                ksel = klast;
+                runsel = runlast;
+                target = INFINITY;
+            }
+            if (ksel < 0) return -1;
+            float v[8], lsum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = 0.f;
+#pragma unroll
+            for (int k = 0; k < ITER; ++k) {
+                if (k == ksel) {          // same for the whole warp
+                    load_stash_t(k, v);
+                    lsum = ls[k];
+                }
+            }
+            float incl = lsum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            float c = runsel + (incl - lsum);
+            int hit = -1, lastp = -1;
+            const int e0 = (wu0 + lane + 32 * ksel) * 8;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                c += v[j];
+                if (v[j] > 0.f) {
+                    lastp = e0 + j;
+                    if (hit < 0 && fmaf(f, c, base) > target) hit = e0 + j;
+                }
+            }
+            const unsigned mh = __ballot_sync(0xFFFFFFFFu, hit >= 0);
+            if (mh) return __shfl_sync(0xFFFFFFFFu, hit, __ffs(mh) - 1);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) lastp = max(lastp, __shfl_xor_sync(0xFFFFFFFFu, lastp, o));
+            return lastp;
+        };
+
+        // ---------------------------------- main loop ----------------------------------------
+        SpecShared* const lead = cluster.map_shared_rank(&sh, 0);
+        if (pcx(0).pos < total) pass_a_any(pcx(0).bonus != 0, true);
+        while (pcx(n).pos < total) {
+            const int par = n & 1;
+            const uint32_t ph = (uint32_t)(n >> 1) & 1u;
+            const bool bonus = pcx(n).bonus != 0;
+            const int npos = pcx(n + 1).pos;
+            const bool nbonus = npos < total && pcx(n + 1).bonus != 0;
+
+            finish_a(bonus);
+            if (bonus) pass_b(std::true_type{});
+            else pass_b(std::false_type{});
+            if (lane == 0) {
+                float4* w = reinterpret_cast<float4*>(&sh.wtab[par][warp]);
+                w[0] = make_float4(Mt_w, sB[0], sB[1], Md_w);
+                w[1] = make_float4(sB[2], sB[3], __uint_as_float(flags_w), 0.f);
+                mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.entry_bar[par]));
+            }
+            __syncwarp();
+            // while the control warps exchange the totals: maxima of the next position, as far
+            // as its slots have landed
+            if (npos < total) pass_a_any(nbonus, false);
+            wait_cta(&sh.scal_bar[par], ph);
+            const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft, base
+            const float4 m1 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp].target); // target, sel
+
+            // pass C: sum (p+q) log2 (p+q) and the overlap indicator sum 2^t_p 2^t_q
+            if (!bonus) {
+                float2 A2 = make_float2(0.f, 0.f), PQ2 = make_float2(0.f, 0.f);
+                const float2 at2 = make_float2(m0.x, m0.x), ad2 = make_float2(m0.y, m0.y);
+                const float2 tiny2 = make_float2(kTiny, kTiny);
+#pragma unroll
+                for (int k = 0; k < ITER; ++k) {
+                    if (k_on(k)) {
+                        float a[8], d[8];
+                        load_stash(k, a, d);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float2 a2 = make_float2(a[2 * j], a[2 * j + 1]);
+                            const float2 d2 = make_float2(d[2 * j], d[2 * j + 1]);
+                            const float2 pp = __ffma2_rn(a2, at2, tiny2);
+                            const float2 ss = __ffma2_rn(d2, ad2, pp);
+                            const float2 ll = make_float2(lg2(ss.x), lg2(ss.y));
+                            A2 = __ffma2_rn(ss, ll, A2);
+                            PQ2 = __ffma2_rn(a2, d2, PQ2);
+                        }
+                    }
+                }
+                const float A = warp_sum(A2.x + A2.y), PQ = warp_sum(PQ2.x + PQ2.y);
+                if (lane == 0) lead->tabC[par][g] = make_float2(A, PQ);
+            }
+            if (__float_as_int(m1.y) != 0) {          // this warp holds the crossing of y_i ~ p_i
+                const int tok = select_kept(m0.w, m0.z, m1.x);
+                if (lane == 0) lead->token[par] = tok;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(reinterpret_cast<uint64_t*>(&sh.c_bar[par]), 0u);
+
+            // the rest of the next position's maxima (waits for slots still in flight)
+            if (npos < total) pass_a_any(nbonus, true);
+            --ip_which;
+            ++n;
+        }
+        // a warp that gave up on a copy still waits (bounded) for whatever it had in flight
+        if (!alive)
+            for (int s = 0; s < NSw; ++s) mbar_wait_bounded(bar_of(s), (phase >> s) & 1u);
+    } else if (warp == kSCtl) {
+        // ============================== control warp ======================================
+        auto sum8 = [&](float v) -> float {       // total of the first eight lanes, in every lane
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+            return __shfl_sync(0xFFFFFFFFu, v, 0);
+        };
+        uint32_t q_head = 0;       // leader: tails pushed so far
+        auto push_tail = [&](int b) {
+            if (lane == 0) {
+                bool room = false;
+                for (uint32_t it = 0; it < kSPollSpins; ++it) {
+                    if (q_head - *reinterpret_cast<volatile uint32_t*>(&sh.tq_tail) < (uint32_t)kSQueue) {
+                        room = true;
+                        break;
+                    }
+                    __nanosleep(100);
+                }
+                if (room) {
+                    reinterpret_cast<volatile int32_t*>(sh.tq)[q_head % kSQueue] = b;
+                    __threadfence_block();
+                    *reinterpret_cast<volatile uint32_t*>(&sh.tq_head) = q_head + 1;
+                } else {
+                    atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                }
+            }
+            ++q_head;
+        };
+        // leader: the published scalars of position number m, once every compute warp of the
+        // cluster has sent its pass-C sums (they did before publishing their next partials)
+        auto finalize = [&](int m) {
+            const int par = m & 1;
+            wait_cluster(&sh.c_bar[par], (uint32_t)(m >> 1) & 1u);
+            const float2 c0 = sh.tabC[par][4 * lane], c1 = sh.tabC[par][4 * lane + 1];
+            const float2 c2 = sh.tabC[par][4 * lane + 2], c3 = sh.tabC[par][4 * lane + 3];
+            const float A = warp_sum(((c0.x + c1.x) + c2.x) + c3.x);
+            const float PQ = warp_sum(((c0.y + c1.y) + c2.y) + c3.y);
+            int done_b = -1;
+            if (lane == 0) {
+                const PosCtx& c = sh.pc[m & (kSPosRing - 1)];
+                const int b = c.pos / K1, i = c.pos - b * K1;
+                const bool bonus = c.bonus != 0;
+                const float Mt = sh.fin[par][0], St = sh.fin[par][1], Tt = sh.fin[par][2];
+                const float Md = sh.fin[par][3], Sd = sh.fin[par][4], Td = sh.fin[par][5];
+                const uint32_t fl = __float_as_uint(sh.fin[par][6]);
+                const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL) || !alive;
+                const size_t idt = (size_t)b * K1 + i, idd = (size_t)b * Kmax + i;
+                int tok = sh.token[par];
+                if (bad) {
+                    atomicOr(p.st.status, ADASD_STATUS_NAN);
+                    tok = -1;
+                }
+                const float lSt = lg2(St), lSd = lg2(Sd);
+                const float Hbt = lSt - Tt / St, Hbd = lSd - Td / Sd;      // entropies in bits
+                float Ht = kLn2 * Hbt, lse_t = kLn2 * (Mt + lSt);
+                if (bad) Ht = lse_t = NAN;
+                p.sc.H_t[idt] = Ht;
+                p.sc.lse_t[idt] = lse_t;
+                p.sc.y[idt] = tok;
+                if (p.user.H_t) p.user.H_t[idt] = Ht;
+                if (p.user.lse_t) p.user.lse_t[idt] = lse_t;
+                if (p.user.y) p.user.y[idt] = tok;
+                if (!bonus) {
+                    float Hd = kLn2 * Hbd, lse_d = kLn2 * (Md + lSd);
+                    // D_JS = H(m) - (H(p) + H(q)) / 2 with H(m) = (ln 2 / 2) (2 - sum s log2 s), s = p + q
+                    float jsd = 0.5f * kLn2 * ((2.f - A) - (Hbt + Hbd));
+                    jsd = (fl & 2u) ? fminf(fmaxf(jsd, 0.f), kLn2) : 0.f;   // identical rows: exactly 0
+                    if (!(PQ > 0.f)) jsd = kLn2;                            // disjoint supports: ln 2
+                    float dist = fminf(sqrtf(jsd / kLn2), 1.f);
+                    if (bad) Hd = lse_d = jsd = dist = NAN;
+                    p.sc.H_d[idd] = Hd;
+                    p.sc.lse_d[idd] = lse_d;
+                    p.sc.jsd[idd] = jsd;
+                    p.sc.dist[idd] = dist;
+                    if (p.user.H_d) p.user.H_d[idd] = Hd;
+                    if (p.user.lse_d) p.user.lse_d[idd] = lse_d;
+                    if (p.user.jsd) p.user.jsd[idd] = jsd;
+                    if (p.user.dist) p.user.dist[idd] = dist;
+                }
+                __threadfence();
+                const unsigned ticket = atomicAdd(p.sc.ticket + b, 1u);
+                if (ticket == (unsigned)c.kt) {
+                    p.sc.ticket[b] = 0u;          // ready for the next round
+                    done_b = b;
+                }
+            }
+            done_b = __shfl_sync(0xFFFFFFFFu, done_b, 0);
+            if (done_b >= 0) push_tail(done_b);
+        };
+
+        int n = 0;
+        while (sh.pc[n & (kSPosRing - 1)].pos < total) {
+            const int par = n & 1;
+            const uint32_t ph = (uint32_t)(n >> 1) & 1u;
+            // describe position n + 3 while the compute warps are busy with position n
+            {
+                PosRef r;
+                r.pos = total;
+                r.kt = 0;
+                if (lastp.pos < total) r = scan_from(lastp.pos + ncl);
+                set_pos(n + 3, r);
+                lastp = r;
+            }
+            const float u_samp = __ldg(p.u_target + sh.pc[n & (kSPosRing - 1)].pos);
+
+            // the CTA's totals from its compute warps, sent to every CTA of the cluster
+            wait_cta(&sh.entry_bar[par], ph);
+            float4 w0 = make_float4(kFloorL, 0.f, 0.f, kFloorL), w1 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (lane < kSW) {
+                const float4* w = reinterpret_cast<const float4*>(&sh.wtab[par][lane]);
+                w0 = w[0];
+                w1 = w[1];
+            }
+            {
+                const float Mt = warp_max_f32(w0.x), Md = warp_max_f32(w0.w);
+                const float dt = w0.x - Mt, dd = w0.w - Md;
+                const float ft = ex2(dt), fd = ex2(dd);
+                const float St = warp_sum(ft * w0.y), Tt = warp_sum(ft * fmaf(dt, w0.y, w0.z));
+                const float Sd = warp_sum(fd * w1.x), Td = warp_sum(fd * fmaf(dd, w1.x, w1.y));
+                const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(w1.z));
+                if (lane < CS) {
+                    float4* dst = reinterpret_cast<float4*>(&cluster.map_shared_rank(&sh, lane)->ctab[par][rank]);
+                    dst[0] = make_float4(Mt, St, Tt, Md);
+                    dst[1] = make_float4(Sd, Td, __uint_as_float(fl), 0.f);
+                    mbar_arrive_remote(reinterpret_cast<uint64_t*>(&sh.ctab_bar[par]), (uint32_t)lane);
+                }
+            }
+            // the row's totals from the CTA totals, lane c holding CTA c
+            wait_cluster(&sh.ctab_bar[par], ph);
+            float4 e0 = make_float4(kFloorL, 0.f, 0.f, kFloorL), e1 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (lane < CS) {
+                const float4* e = reinterpret_cast<const float4*>(&sh.ctab[par][lane]);
+                e0 = e[0];
+                e1 = e[1];
+            }
+            const float Mt = warp_max_f32(e0.x), Md = warp_max_f32(e0.w);
+            const float cdt = e0.x - Mt, cdd = e0.w - Md;
+            const float cft = ex2(cdt), cfd = ex2(cdd);
+            const float st_c = cft * e0.y;                    // CTA sums of the target row, scaled to Mt
+            const float St = sum8(st_c), Sd = sum8(cfd * e1.x);
+            const float Tt = sum8(cft * fmaf(cdt, e0.y, e0.z)), Td = sum8(cfd * fmaf(cdd, e1.x, e1.y));
+            const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(e1.z));
+            const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL);
+
+            // one message per compute warp (lane w): its scale factors, and whether it holds the
+            // crossing of target = u * S_t in index order (CTA by CTA, then warp by warp)
+            const float ftw = ex2(w0.x - Mt), fdw = ex2(w0.w - Md);
+            const float at = ftw / St, ad = fdw / Sd;
+            int sel = 0;
+            float base = 0.f, target = u_samp * St;
+            if (!bad) {
+                float incl = st_c;
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) {
+                    const float t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const bool mass = lane < CS && st_c > 0.f;
+                int cstar = -1;
+                const unsigned mc = __ballot_sync(0xFFFFFFFFu, mass && incl > target);
+                if (mc) {
+                    cstar = __ffs(mc) - 1;
+                } else {
+                    const unsigned ml = __ballot_sync(0xFFFFFFFFu, mass);
+                    if (ml) cstar = 31 - __clz(ml);
+                    target = INFINITY;
+                }
+                const float cbase = __shfl_sync(0xFFFFFFFFu, incl - st_c, max(cstar, 0));
+                if (cstar == rank) {
+                    const float w = (lane < kSW) ? ftw * w0.y : 0.f;
+                    float winc = w;
+#pragma unroll
+                    for (int o = 1; o < 16; o <<= 1) {
+                        const float t = __shfl_up_sync(0xFFFFFFFFu, winc, o);
+                        if (lane >= o) winc += t;
+                    }
+                    int wsel = -1;
+                    const unsigned mh = __ballot_sync(0xFFFFFFFFu, w > 0.f && cbase + winc > target);
+                    if (mh) {
+                        wsel = __ffs(mh) - 1;
+                    } else {
+                        const unsigned ml = __ballot_sync(0xFFFFFFFFu, w > 0.f);
+                        if (ml) wsel = 31 - __clz(ml);
+                        target = INFINITY;
+                    }
+                    if (lane == wsel) {
+                        sel = 1;
+                        base = cbase + (winc - w);
+                    }
+                }
+            }
+            if (lane < kSW) {
+                float4* m = reinterpret_cast<float4*>(&sh.wmsg[par][lane]);
+                m[0] = make_float4(at, ad, ftw, base);
+                m[1] = make_float4(target, __int_as_float(sel), 0.f, 0.f);
+            }
+            if (leader && lane == 0) {
+                sh.fin[par][0] = Mt;
+                sh.fin[par][1] = St;
+                sh.fin[par][2] = Tt;
+                sh.fin[par][3] = Md;
+                sh.fin[par][4] = Sd;
+                sh.fin[par][5] = Td;
+                sh.fin[par][6] = __uint_as_float(fl | (alive ? 0u : 1u));
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.scal_bar[par]));
+
+            if (leader && n > 0) finalize(n - 1);
+            ++n;
+        }
+        if (leader) {
+            if (n > 0) finalize(n - 1);
+            push_tail(-1);
+        }
+    } else {
+        // ================================ tail warp =======================================
+        if (leader) {
+            TailIO io;
+            io.H_d = p.sc.H_d;
+            io.dist = p.sc.dist;
+            io.y = p.sc.y;
+            io.x = p.x;
+            io.u_accept = p.u_accept;
+            io.draft_len = p.draft_len;
+            io.p_acc = p.sc.p_acc;
+            io.p_acc_user = p.user.p_acc;
+            io.accept_len = p.accept_len;
+            io.next_token = p.next_token;
+            io.accept_len_rec = p.user.accept_len;
+            io.rejected_rec = p.user.rejected;
+            io.draft_len_rec = p.user.draft_len;
+            for (uint32_t t = 0;; ++t) {
+                int b = -2;
+                if (lane == 0) {
+                    for (uint32_t it = 0; it < kSPollSpins; ++it) {
+                        if (*reinterpret_cast<volatile uint32_t*>(&sh.tq_head) != t) {
+                            __threadfence_block();
+                            b = reinterpret_cast<volatile int32_t*>(sh.tq)[t % kSQueue];
+                            break;
+                        }
+                        __nanosleep(200);
+                    }
+                    if (b == -2) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                }
+                b = __shfl_sync(0xFFFFFFFFu, b, 0);
+                if (b < 0) break;            // stop mark, or the queue never filled
+                __threadfence();
+                verify_tail_warp(p.tail, io, p.st, b, sh.td, sh.tH);
+                if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&sh.tq_tail) = t + 1;
+            }
+        }
+    }
+    cluster.sync();   // no CTA leaves while a peer may still address its shared memory
+}
+
+}  // namespace adasd
