@@ -30,9 +30,9 @@ constexpr int kSTail = kSW + 1;                  // warp index of the tail warp
 constexpr int kSThreads = (kSW + 2) * 32;        // 384: leaves 168 registers per thread
 constexpr int kSRegIter = 6;                     // iterations whose 2^t values stay in registers
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
-constexpr int kSPosRing = 8;                     // positions the control warp keeps described
-constexpr int kSQueue = 64;                      // tail queue entries
-constexpr uint32_t kSPollSpins = 1u << 24;       // polls of the tail queue before giving up
+constexpr int kSPosRing = 16;                    // positions the control warp keeps described
+constexpr int kSFinRing = 8;                     // positions whose sums may await finalisation
+constexpr uint32_t kSPollSpins = 1u << 24;       // polls of a progress counter before giving up
 
 // One position as the control warp describes it to the compute warps of its CTA.
 struct __align__(16) PosCtx {
@@ -58,16 +58,17 @@ struct __align__(16) SpecShared {
     RowPart wtab[2][kCW];             // this CTA's compute warps, by position parity
     RowPart ctab[2][kCMaxCluster];    // every CTA's totals (written over DSMEM), by parity
     WarpMsg wmsg[2][kCW];
-    float2 tabC[2][kCTab];            // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q)
-    float fin[2][8];                  // leader: row totals kept for finalisation
-    int32_t token[2];                 // leader: sampled token of the position
+    float2 tabC[kSFinRing][kCTab];    // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q), by position & 7
+    float fin[kSFinRing][8];          // leader: row totals kept for finalisation
+    int32_t token[kSFinRing];         // leader: sampled token of the position
     unsigned long long entry_bar[2];  // one arrival per compute warp: wtab[par] complete
     unsigned long long ctab_bar[2];   // CS remote arrivals: ctab[par] complete
     unsigned long long scal_bar[2];   // 1 arrival: wmsg[par] ready
-    unsigned long long c_bar[2];      // leader: one remote arrival per compute warp of the cluster: tabC[par], token[par] complete
+    unsigned long long c_bar[kSFinRing];   // leader: one remote arrival per compute warp of the cluster: tabC, token complete
     unsigned long long bar[kCW][kCMaxSlots];   // "slot filled" barriers
-    int32_t tq[kSQueue];              // leader: sequences whose tail must run (-1: stop)
-    uint32_t tq_head, tq_tail;        // pushed by the control warp / done by the tail warp
+    int32_t n_issued;                 // leader: positions whose messages have been sent
+    int32_t n_final;                  // leader: number of positions of this cluster, -1 until known
+    int32_t fin_done;                 // leader: positions finalised so far (written by the tail warp)
     float td[ADASD_KMAX_LIMIT], tH[ADASD_KMAX_LIMIT];   // tail warp scratch
 };
 
@@ -245,19 +246,23 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
     const int NU = p.V >> 3;                                   // 16-byte units per row
     const int cu0 = (int)((long long)rank * NU / CS), cu1 = (int)((long long)(rank + 1) * NU / CS);
 
-    for (int q = threadIdx.x; q < 4 * kCTab; q += kSThreads) reinterpret_cast<float*>(sh.tabC)[q] = 0.f;
+    for (int q = threadIdx.x; q < 2 * kSFinRing * kCTab; q += kSThreads) reinterpret_cast<float*>(sh.tabC)[q] = 0.f;
     if (threadIdx.x < kSPosRing) {
         sh.pc[threadIdx.x].pos = total;
         sh.pc[threadIdx.x].kt = 0;
         sh.pc[threadIdx.x].bonus = 0;
     }
     if (threadIdx.x == 0) {
-        sh.token[0] = sh.token[1] = -1;
-        sh.tq_head = sh.tq_tail = 0u;
+        sh.n_issued = 0;
+        sh.n_final = -1;
+        sh.fin_done = 0;
         for (int k = 0; k < 2; ++k) {
             mbar_init(reinterpret_cast<uint64_t*>(&sh.entry_bar[k]), kSW);
             mbar_init(reinterpret_cast<uint64_t*>(&sh.ctab_bar[k]), (uint32_t)CS);
             mbar_init(reinterpret_cast<uint64_t*>(&sh.scal_bar[k]), 1);
+        }
+        for (int k = 0; k < kSFinRing; ++k) {
+            sh.token[k] = -1;
             mbar_init(reinterpret_cast<uint64_t*>(&sh.c_bar[k]), (uint32_t)(CS * kSW));
         }
     }
@@ -697,14 +702,14 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     }
                 }
                 const float A = warp_sum(A2.x + A2.y), PQ = warp_sum(PQ2.x + PQ2.y);
-                if (lane == 0) lead->tabC[par][g] = make_float2(A, PQ);
+                if (lane == 0) lead->tabC[n & (kSFinRing - 1)][g] = make_float2(A, PQ);
             }
             if (__float_as_int(m1.y) != 0) {          // this warp holds the crossing of y_i ~ p_i
                 const int tok = select_kept(m0.w, m0.z, m1.x);
-                if (lane == 0) lead->token[par] = tok;
+                if (lane == 0) lead->token[n & (kSFinRing - 1)] = tok;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(reinterpret_cast<uint64_t*>(&sh.c_bar[par]), 0u);
+            if (lane == 0) mbar_arrive_remote(reinterpret_cast<uint64_t*>(&sh.c_bar[n & (kSFinRing - 1)]), 0u);
 
             // the rest of the next position's maxima (waits for slots still in flight)
             if (npos < total) pass_a_any(nbonus, true);
@@ -722,89 +727,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
             return __shfl_sync(0xFFFFFFFFu, v, 0);
         };
-        uint32_t q_head = 0;       // leader: tails pushed so far
-        auto push_tail = [&](int b) {
-            if (lane == 0) {
-                bool room = false;
-                for (uint32_t it = 0; it < kSPollSpins; ++it) {
-                    if (q_head - *reinterpret_cast<volatile uint32_t*>(&sh.tq_tail) < (uint32_t)kSQueue) {
-                        room = true;
-                        break;
-                    }
-                    __nanosleep(100);
-                }
-                if (room) {
-                    reinterpret_cast<volatile int32_t*>(sh.tq)[q_head % kSQueue] = b;
-                    __threadfence_block();
-                    *reinterpret_cast<volatile uint32_t*>(&sh.tq_head) = q_head + 1;
-                } else {
-                    atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
-                }
-            }
-            ++q_head;
-        };
-        // leader: the published scalars of position number m, once every compute warp of the
-        // cluster has sent its pass-C sums (they did before publishing their next partials)
-        auto finalize = [&](int m) {
-            const int par = m & 1;
-            wait_cluster(&sh.c_bar[par], (uint32_t)(m >> 1) & 1u);
-            const float2 c0 = sh.tabC[par][4 * lane], c1 = sh.tabC[par][4 * lane + 1];
-            const float2 c2 = sh.tabC[par][4 * lane + 2], c3 = sh.tabC[par][4 * lane + 3];
-            const float A = warp_sum(((c0.x + c1.x) + c2.x) + c3.x);
-            const float PQ = warp_sum(((c0.y + c1.y) + c2.y) + c3.y);
-            int done_b = -1;
-            if (lane == 0) {
-                const PosCtx& c = sh.pc[m & (kSPosRing - 1)];
-                const int b = c.pos / K1, i = c.pos - b * K1;
-                const bool bonus = c.bonus != 0;
-                const float Mt = sh.fin[par][0], St = sh.fin[par][1], Tt = sh.fin[par][2];
-                const float Md = sh.fin[par][3], Sd = sh.fin[par][4], Td = sh.fin[par][5];
-                const uint32_t fl = __float_as_uint(sh.fin[par][6]);
-                const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL) || !alive;
-                const size_t idt = (size_t)b * K1 + i, idd = (size_t)b * Kmax + i;
-                int tok = sh.token[par];
-                if (bad) {
-                    atomicOr(p.st.status, ADASD_STATUS_NAN);
-                    tok = -1;
-                }
-                const float lSt = lg2(St), lSd = lg2(Sd);
-                const float Hbt = lSt - Tt / St, Hbd = lSd - Td / Sd;      // entropies in bits
-                float Ht = kLn2 * Hbt, lse_t = kLn2 * (Mt + lSt);
-                if (bad) Ht = lse_t = NAN;
-                p.sc.H_t[idt] = Ht;
-                p.sc.lse_t[idt] = lse_t;
-                p.sc.y[idt] = tok;
-                if (p.user.H_t) p.user.H_t[idt] = Ht;
-                if (p.user.lse_t) p.user.lse_t[idt] = lse_t;
-                if (p.user.y) p.user.y[idt] = tok;
-                if (!bonus) {
-                    float Hd = kLn2 * Hbd, lse_d = kLn2 * (Md + lSd);
-                    // D_JS = H(m) - (H(p) + H(q)) / 2 with H(m) = (ln 2 / 2) (2 - sum s log2 s), s = p + q
-                    float jsd = 0.5f * kLn2 * ((2.f - A) - (Hbt + Hbd));
-                    jsd = (fl & 2u) ? fminf(fmaxf(jsd, 0.f), kLn2) : 0.f;   // identical rows: exactly 0
-                    if (!(PQ > 0.f)) jsd = kLn2;                            // disjoint supports: ln 2
-                    float dist = fminf(sqrtf(jsd / kLn2), 1.f);
-                    if (bad) Hd = lse_d = jsd = dist = NAN;
-                    p.sc.H_d[idd] = Hd;
-                    p.sc.lse_d[idd] = lse_d;
-                    p.sc.jsd[idd] = jsd;
-                    p.sc.dist[idd] = dist;
-                    if (p.user.H_d) p.user.H_d[idd] = Hd;
-                    if (p.user.lse_d) p.user.lse_d[idd] = lse_d;
-                    if (p.user.jsd) p.user.jsd[idd] = jsd;
-                    if (p.user.dist) p.user.dist[idd] = dist;
-                }
-                __threadfence();
-                const unsigned ticket = atomicAdd(p.sc.ticket + b, 1u);
-                if (ticket == (unsigned)c.kt) {
-                    p.sc.ticket[b] = 0u;          // ready for the next round
-                    done_b = b;
-                }
-            }
-            done_b = __shfl_sync(0xFFFFFFFFu, done_b, 0);
-            if (done_b >= 0) push_tail(done_b);
-        };
-
         int n = 0;
         while (sh.pc[n & (kSPosRing - 1)].pos < total) {
             const int par = n & 1;
@@ -822,6 +744,17 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
 
             // the CTA's totals from its compute warps, sent to every CTA of the cluster
             wait_cta(&sh.entry_bar[par], ph);
+            if (leader && lane == 0) {
+                // before anybody can send sums of position n: the ring entry it reuses (position
+                // n - kSFinRing) must have been finalised
+                bool room = !alive;
+                for (uint32_t it = 0; !room && it < kSPollSpins; ++it) {
+                    room = *reinterpret_cast<volatile int32_t*>(&sh.fin_done) > n - kSFinRing;
+                    if (!room) __nanosleep(100);
+                }
+                if (!room) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+            }
+            __syncwarp();
             float4 w0 = make_float4(kFloorL, 0.f, 0.f, kFloorL), w1 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (lane < kSW) {
                 const float4* w = reinterpret_cast<const float4*>(&sh.wtab[par][lane]);
@@ -912,26 +845,30 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 m[1] = make_float4(target, __int_as_float(sel), 0.f, 0.f);
             }
             if (leader && lane == 0) {
-                sh.fin[par][0] = Mt;
-                sh.fin[par][1] = St;
-                sh.fin[par][2] = Tt;
-                sh.fin[par][3] = Md;
-                sh.fin[par][4] = Sd;
-                sh.fin[par][5] = Td;
-                sh.fin[par][6] = __uint_as_float(fl | (alive ? 0u : 1u));
+                float* f = sh.fin[n & (kSFinRing - 1)];
+                f[0] = Mt;
+                f[1] = St;
+                f[2] = Tt;
+                f[3] = Md;
+                f[4] = Sd;
+                f[5] = Td;
+                f[6] = __uint_as_float(fl | (alive ? 0u : 1u));
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.scal_bar[par]));
-
-            if (leader && n > 0) finalize(n - 1);
+            if (lane == 0) {
+                mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.scal_bar[par]));
+                if (leader) *reinterpret_cast<volatile int32_t*>(&sh.n_issued) = n + 1;
+            }
             ++n;
         }
-        if (leader) {
-            if (n > 0) finalize(n - 1);
-            push_tail(-1);
+        if (leader && lane == 0) {
+            __threadfence_block();
+            *reinterpret_cast<volatile int32_t*>(&sh.n_final) = n;
         }
     } else {
         // ================================ tail warp =======================================
+        // Leader CTA only: finalises every position of the cluster, in order, as soon as its sums
+        // are in, and runs the tail of each sequence whose last position that was.
         if (leader) {
             TailIO io;
             io.H_d = p.sc.H_d;
@@ -947,24 +884,96 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             io.accept_len_rec = p.user.accept_len;
             io.rejected_rec = p.user.rejected;
             io.draft_len_rec = p.user.draft_len;
-            for (uint32_t t = 0;; ++t) {
-                int b = -2;
+            // leader: the published scalars of position number m, once every compute warp of the
+            // cluster has sent its pass-C sums (they did before publishing their next partials)
+            auto finalize = [&](int m) -> int {
+                const int par = m & (kSFinRing - 1);
+                wait_cluster(&sh.c_bar[par], (uint32_t)(m / kSFinRing) & 1u);
+                const float2 c0 = sh.tabC[par][4 * lane], c1 = sh.tabC[par][4 * lane + 1];
+                const float2 c2 = sh.tabC[par][4 * lane + 2], c3 = sh.tabC[par][4 * lane + 3];
+                const float A = warp_sum(((c0.x + c1.x) + c2.x) + c3.x);
+                const float PQ = warp_sum(((c0.y + c1.y) + c2.y) + c3.y);
+                int done_b = -1;
+                if (lane == 0) {
+                    const PosCtx& c = sh.pc[m & (kSPosRing - 1)];
+                    const int b = c.pos / K1, i = c.pos - b * K1;
+                    const bool bonus = c.bonus != 0;
+                    const float Mt = sh.fin[par][0], St = sh.fin[par][1], Tt = sh.fin[par][2];
+                    const float Md = sh.fin[par][3], Sd = sh.fin[par][4], Td = sh.fin[par][5];
+                    const uint32_t fl = __float_as_uint(sh.fin[par][6]);
+                    const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL) || !alive;
+                    const size_t idt = (size_t)b * K1 + i, idd = (size_t)b * Kmax + i;
+                    int tok = sh.token[par];
+                    if (bad) {
+                        atomicOr(p.st.status, ADASD_STATUS_NAN);
+                        tok = -1;
+                    }
+                    const float lSt = lg2(St), lSd = lg2(Sd);
+                    const float Hbt = lSt - Tt / St, Hbd = lSd - Td / Sd;      // entropies in bits
+                    float Ht = kLn2 * Hbt, lse_t = kLn2 * (Mt + lSt);
+                    if (bad) Ht = lse_t = NAN;
+                    p.sc.H_t[idt] = Ht;
+                    p.sc.lse_t[idt] = lse_t;
+                    p.sc.y[idt] = tok;
+                    if (p.user.H_t) p.user.H_t[idt] = Ht;
+                    if (p.user.lse_t) p.user.lse_t[idt] = lse_t;
+                    if (p.user.y) p.user.y[idt] = tok;
+                    if (!bonus) {
+                        float Hd = kLn2 * Hbd, lse_d = kLn2 * (Md + lSd);
+                        // D_JS = H(m) - (H(p) + H(q)) / 2 with H(m) = (ln 2 / 2) (2 - sum s log2 s), s = p + q
+                        float jsd = 0.5f * kLn2 * ((2.f - A) - (Hbt + Hbd));
+                        jsd = (fl & 2u) ? fminf(fmaxf(jsd, 0.f), kLn2) : 0.f;   // identical rows: exactly 0
+                        if (!(PQ > 0.f)) jsd = kLn2;                            // disjoint supports: ln 2
+                        float dist = fminf(sqrtf(jsd / kLn2), 1.f);
+                        if (bad) Hd = lse_d = jsd = dist = NAN;
+                        p.sc.H_d[idd] = Hd;
+                        p.sc.lse_d[idd] = lse_d;
+                        p.sc.jsd[idd] = jsd;
+                        p.sc.dist[idd] = dist;
+                        if (p.user.H_d) p.user.H_d[idd] = Hd;
+                        if (p.user.lse_d) p.user.lse_d[idd] = lse_d;
+                        if (p.user.jsd) p.user.jsd[idd] = jsd;
+                        if (p.user.dist) p.user.dist[idd] = dist;
+                    }
+                    __threadfence();
+                    const unsigned ticket = atomicAdd(p.sc.ticket + b, 1u);
+                    if (ticket == (unsigned)c.kt) {
+                        p.sc.ticket[b] = 0u;          // ready for the next round
+                        done_b = b;
+                    }
+                }
+                return __shfl_sync(0xFFFFFFFFu, done_b, 0);
+            };
+
+            for (int m = 0;; ++m) {
+                // position m exists once its messages have gone out; the control warp says when
+                // the cluster has no more
+                int go = -1;
                 if (lane == 0) {
                     for (uint32_t it = 0; it < kSPollSpins; ++it) {
-                        if (*reinterpret_cast<volatile uint32_t*>(&sh.tq_head) != t) {
-                            __threadfence_block();
-                            b = reinterpret_cast<volatile int32_t*>(sh.tq)[t % kSQueue];
+                        if (*reinterpret_cast<volatile int32_t*>(&sh.n_issued) > m) {
+                            go = 1;
                             break;
                         }
-                        __nanosleep(200);
+                        if (*reinterpret_cast<volatile int32_t*>(&sh.n_final) == m) {
+                            go = 0;
+                            break;
+                        }
+                        __nanosleep(100);
                     }
-                    if (b == -2) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                    if (go < 0) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
                 }
-                b = __shfl_sync(0xFFFFFFFFu, b, 0);
-                if (b < 0) break;            // stop mark, or the queue never filled
-                __threadfence();
-                verify_tail_warp(p.tail, io, p.st, b, sh.td, sh.tH);
-                if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&sh.tq_tail) = t + 1;
+                go = __shfl_sync(0xFFFFFFFFu, go, 0);
+                if (go <= 0) break;
+                const int done_b = finalize(m);
+                if (done_b >= 0) {
+                    __threadfence();
+                    verify_tail_warp(p.tail, io, p.st, done_b, sh.td, sh.tH);
+                }
+                if (lane == 0) {
+                    __threadfence_block();
+                    *reinterpret_cast<volatile int32_t*>(&sh.fin_done) = m + 1;
+                }
             }
         }
     }
