@@ -8,12 +8,13 @@
 //    (maxima; 2^t, S and T; (p+q) log2 (p+q)), the refill of their own ring slots and, for
 //    the one warp that holds it, the inverse-CDF crossing.
 //  * 1 CONTROL warp per CTA finds the cluster's positions, folds the warp partials into the
-//    CTA's totals, exchanges them with the other CTAs of the cluster (DSMEM stores + remote
-//    mbarrier arrivals: no cluster-wide barrier in the loop), turns the row totals into one
-//    small message per compute warp (its scale factors and whether it holds the crossing) and,
-//    in the leader CTA, finalises the previous position and draws the sequence's ticket.
-//  * 1 TAIL warp per CTA runs the tails (KDE/Bayes, accept scan, list appends, T_G) of the
-//    sequences its control warp completes, off everybody's critical path.
+//    CTA's totals, exchanges them with the other CTAs of the cluster (st.async into their
+//    shared memory, counted on their mbarriers: no cluster-wide barrier in the loop) and
+//    turns the row totals into two small messages per compute warp: its scale factors, then
+//    whether it holds the inverse-CDF crossing.
+//  * 1 TAIL warp (leader CTA) finalises each position once the compute warps' sums are in,
+//    draws the sequence's ticket and runs the tails (KDE/Bayes, accept scan, list appends,
+//    T_G) of completed sequences, off everybody's critical path.
 //
 // Every wait (slot filled, partials in, totals in, message ready, sums in, queue) is bounded:
 // a warp whose wait expires sets ADASD_STATUS_TIMEOUT, stops waiting and copying, and walks
@@ -31,7 +32,7 @@ constexpr int kSThreads = (kSW + 2) * 32;        // 384: leaves 168 registers pe
 constexpr int kSRegIter = 6;                     // iterations whose 2^t values stay in registers
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
 constexpr int kSPosRing = 16;                    // positions the control warp keeps described
-constexpr int kSFinRing = 8;                     // positions whose sums may await finalisation
+constexpr int kSFinRing = 4;                     // positions whose sums may await finalisation
 constexpr uint32_t kSPollSpins = 1u << 24;       // polls of a progress counter before giving up
 
 // One position as the control warp describes it to the compute warps of its CTA.
@@ -47,10 +48,11 @@ struct __align__(16) PosCtx {
 // What a compute warp needs after the exchange: p = 2^t_p * at, q = 2^t_q * ad; and, if it
 // holds the inverse-CDF crossing (sel), the weight before its share and the target.
 struct __align__(16) WarpMsg {
-    float at, ad, ft, base;
-    float target;
+    float at, ad, ft, pad0;       // first part: ready when scal_bar completes
+    float target;                 // second part: ready when sel_bar completes
     int32_t sel;
-    int32_t pad0, pad1;
+    float base;
+    int32_t pad1;
 };
 
 struct __align__(16) SpecShared {
@@ -58,13 +60,13 @@ struct __align__(16) SpecShared {
     RowPart wtab[2][kCW];             // this CTA's compute warps, by position parity
     RowPart ctab[2][kCMaxCluster];    // every CTA's totals (written over DSMEM), by parity
     WarpMsg wmsg[2][kCW];
-    float2 tabC[kSFinRing][kCTab];    // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q), by position & 7
+    float4 tabC[kSFinRing][kCTab];    // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q, token or -1), by position
     float fin[kSFinRing][8];          // leader: row totals kept for finalisation
-    int32_t token[kSFinRing];         // leader: sampled token of the position
     unsigned long long entry_bar[2];  // one arrival per compute warp: wtab[par] complete
-    unsigned long long ctab_bar[2];   // CS remote arrivals: ctab[par] complete
-    unsigned long long scal_bar[2];   // 1 arrival: wmsg[par] ready
-    unsigned long long c_bar[kSFinRing];   // leader: one remote arrival per compute warp of the cluster: tabC, token complete
+    unsigned long long ctab_bar[2];   // CS * 32 bytes from the control warps of the cluster: ctab[par] complete
+    unsigned long long scal_bar[2];   // 1 arrival: first part of wmsg[par] ready
+    unsigned long long sel_bar[2];    // 1 arrival: second part of wmsg[par] ready
+    unsigned long long c_bar[kSFinRing];   // leader: 16 bytes from every compute warp of the cluster: tabC complete
     unsigned long long bar[kCW][kCMaxSlots];   // "slot filled" barriers
     int32_t n_issued;                 // leader: positions whose messages have been sent
     int32_t n_final;                  // leader: number of positions of this cluster, -1 until known
@@ -76,31 +78,18 @@ struct __align__(16) SpecShared {
 __device__ __forceinline__ void mbar_arrive_cta(uint64_t* bar) {
     asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// arrival on the same barrier in CTA `cta` of the cluster; releases this thread's earlier
-// writes (its DSMEM stores included) to whoever acquires at cluster scope
-__device__ __forceinline__ void mbar_arrive_remote(uint64_t* bar, uint32_t cta) {
-    asm volatile(
-        "{\n\t.reg .b32 ra;\n\t"
-        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
-        ::"r"(smem_u32(bar)), "r"(cta)
-        : "memory");
+// shared::cluster address of `p` (an address in this CTA's shared memory) as seen in CTA `cta`
+__device__ __forceinline__ uint32_t mapa_u32(const void* p, uint32_t cta) {
+    uint32_t r;
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(cta));
+    return r;
 }
-__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kCWaitSpins; ++it)
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-    return false;
+// 16 bytes into another CTA's shared memory; their arrival is counted (complete_tx) on a
+// barrier of THAT CTA, so the receiver needs no fence and the sender no second message
+__device__ __forceinline__ void st_async_v4(uint32_t remote_addr, float4 v, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(remote_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar)
+                 : "memory");
 }
 
 // The per-sequence tail of a round, run by ONE warp: lane i owns candidate i.  Same
@@ -246,7 +235,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
     const int NU = p.V >> 3;                                   // 16-byte units per row
     const int cu0 = (int)((long long)rank * NU / CS), cu1 = (int)((long long)(rank + 1) * NU / CS);
 
-    for (int q = threadIdx.x; q < 2 * kSFinRing * kCTab; q += kSThreads) reinterpret_cast<float*>(sh.tabC)[q] = 0.f;
+    for (int q = threadIdx.x; q < kSFinRing * kCTab; q += kSThreads)
+        reinterpret_cast<float4*>(sh.tabC)[q] = make_float4(0.f, 0.f, __int_as_float(-1), 0.f);
     if (threadIdx.x < kSPosRing) {
         sh.pc[threadIdx.x].pos = total;
         sh.pc[threadIdx.x].kt = 0;
@@ -258,13 +248,11 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         sh.fin_done = 0;
         for (int k = 0; k < 2; ++k) {
             mbar_init(reinterpret_cast<uint64_t*>(&sh.entry_bar[k]), kSW);
-            mbar_init(reinterpret_cast<uint64_t*>(&sh.ctab_bar[k]), (uint32_t)CS);
+            mbar_init(reinterpret_cast<uint64_t*>(&sh.ctab_bar[k]), 1);
             mbar_init(reinterpret_cast<uint64_t*>(&sh.scal_bar[k]), 1);
+            mbar_init(reinterpret_cast<uint64_t*>(&sh.sel_bar[k]), 1);
         }
-        for (int k = 0; k < kSFinRing; ++k) {
-            sh.token[k] = -1;
-            mbar_init(reinterpret_cast<uint64_t*>(&sh.c_bar[k]), (uint32_t)(CS * kSW));
-        }
+        for (int k = 0; k < kSFinRing; ++k) mbar_init(reinterpret_cast<uint64_t*>(&sh.c_bar[k]), 1);
     }
     if (warp < kSW && lane == 0)
         for (int s = 0; s < kCMaxSlots; ++s) mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][s]), 1);
@@ -338,12 +326,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
     auto wait_cta = [&](unsigned long long* bar, uint32_t par) {
         if (!alive) return;
         bool ok = mbar_wait_bounded(reinterpret_cast<uint64_t*>(bar), par);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) expired();
-    };
-    auto wait_cluster = [&](unsigned long long* bar, uint32_t par) {
-        if (!alive) return;
-        bool ok = mbar_wait_bounded_cluster(reinterpret_cast<uint64_t*>(bar), par);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) expired();
     };
@@ -653,7 +635,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         };
 
         // ---------------------------------- main loop ----------------------------------------
-        SpecShared* const lead = cluster.map_shared_rank(&sh, 0);
         if (pcx(0).pos < total) pass_a_any(pcx(0).bonus != 0, true);
         while (pcx(n).pos < total) {
             const int par = n & 1;
@@ -676,10 +657,10 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             // as its slots have landed
             if (npos < total) pass_a_any(nbonus, false);
             wait_cta(&sh.scal_bar[par], ph);
-            const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft, base
-            const float4 m1 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp].target); // target, sel
+            const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft
 
             // pass C: sum (p+q) log2 (p+q) and the overlap indicator sum 2^t_p 2^t_q
+            float A = 0.f, PQ = 0.f;
             if (!bonus) {
                 float2 A2 = make_float2(0.f, 0.f), PQ2 = make_float2(0.f, 0.f);
                 const float2 at2 = make_float2(m0.x, m0.x), ad2 = make_float2(m0.y, m0.y);
@@ -701,15 +682,22 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                         }
                     }
                 }
-                const float A = warp_sum(A2.x + A2.y), PQ = warp_sum(PQ2.x + PQ2.y);
-                if (lane == 0) lead->tabC[n & (kSFinRing - 1)][g] = make_float2(A, PQ);
+                A = warp_sum(A2.x + A2.y);
+                PQ = warp_sum(PQ2.x + PQ2.y);
             }
-            if (__float_as_int(m1.y) != 0) {          // this warp holds the crossing of y_i ~ p_i
-                const int tok = select_kept(m0.w, m0.z, m1.x);
-                if (lane == 0) lead->token[n & (kSFinRing - 1)] = tok;
+            // y_i ~ p_i: the control warp says (a little later than the scale factors) whether this
+            // warp holds the crossing
+            wait_cta(&sh.sel_bar[par], ph);
+            const float4 m1 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp].target); // target, sel, base
+            int tok = -1;
+            if (__float_as_int(m1.y) != 0) tok = select_kept(m1.z, m0.z, m1.x);
+            // this warp's sums (and the token, if it drew it) go to the leader CTA in one message
+            if (lane == 0) {
+                const int fr = n & (kSFinRing - 1);
+                st_async_v4(mapa_u32(&sh.tabC[fr][g], 0u), make_float4(A, PQ, __int_as_float(tok), 0.f),
+                            mapa_u32(&sh.c_bar[fr], 0u));
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(reinterpret_cast<uint64_t*>(&sh.c_bar[n & (kSFinRing - 1)]), 0u);
 
             // the rest of the next position's maxima (waits for slots still in flight)
             if (npos < total) pass_a_any(nbonus, true);
@@ -753,6 +741,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     if (!room) __nanosleep(100);
                 }
                 if (!room) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                // every compute warp of the cluster will send 16 bytes for position n
+                mbar_expect_tx(reinterpret_cast<uint64_t*>(&sh.c_bar[n & (kSFinRing - 1)]), (uint32_t)(CS * kSW * 16));
             }
             __syncwarp();
             float4 w0 = make_float4(kFloorL, 0.f, 0.f, kFloorL), w1 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -768,15 +758,16 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 const float St = warp_sum(ft * w0.y), Tt = warp_sum(ft * fmaf(dt, w0.y, w0.z));
                 const float Sd = warp_sum(fd * w1.x), Td = warp_sum(fd * fmaf(dd, w1.x, w1.y));
                 const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(w1.z));
+                if (lane == 0) mbar_expect_tx(reinterpret_cast<uint64_t*>(&sh.ctab_bar[par]), (uint32_t)(CS * 32));
                 if (lane < CS) {
-                    float4* dst = reinterpret_cast<float4*>(&cluster.map_shared_rank(&sh, lane)->ctab[par][rank]);
-                    dst[0] = make_float4(Mt, St, Tt, Md);
-                    dst[1] = make_float4(Sd, Td, __uint_as_float(fl), 0.f);
-                    mbar_arrive_remote(reinterpret_cast<uint64_t*>(&sh.ctab_bar[par]), (uint32_t)lane);
+                    const uint32_t dst = mapa_u32(&sh.ctab[par][rank], (uint32_t)lane);
+                    const uint32_t bar = mapa_u32(&sh.ctab_bar[par], (uint32_t)lane);
+                    st_async_v4(dst, make_float4(Mt, St, Tt, Md), bar);
+                    st_async_v4(dst + 16, make_float4(Sd, Td, __uint_as_float(fl), 0.f), bar);
                 }
             }
             // the row's totals from the CTA totals, lane c holding CTA c
-            wait_cluster(&sh.ctab_bar[par], ph);
+            wait_cta(&sh.ctab_bar[par], ph);
             float4 e0 = make_float4(kFloorL, 0.f, 0.f, kFloorL), e1 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (lane < CS) {
                 const float4* e = reinterpret_cast<const float4*>(&sh.ctab[par][lane]);
@@ -788,14 +779,20 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const float cft = ex2(cdt), cfd = ex2(cdd);
             const float st_c = cft * e0.y;                    // CTA sums of the target row, scaled to Mt
             const float St = sum8(st_c), Sd = sum8(cfd * e1.x);
+
+            // first message per compute warp (lane w): its scale factors; pass C starts on it
+            const float ftw = ex2(w0.x - Mt), fdw = ex2(w0.w - Md);
+            const float at = __fdividef(ftw, St), ad = __fdividef(fdw, Sd);
+            if (lane < kSW) *reinterpret_cast<float4*>(&sh.wmsg[par][lane]) = make_float4(at, ad, ftw, 0.f);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.scal_bar[par]));
+
+            // off the critical path: T totals and flags for the finaliser, then the second message:
+            // which warp holds the crossing of target = u * S_t in index order (CTA by CTA, then
+            // warp by warp)
             const float Tt = sum8(cft * fmaf(cdt, e0.y, e0.z)), Td = sum8(cfd * fmaf(cdd, e1.x, e1.y));
             const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(e1.z));
             const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL);
-
-            // one message per compute warp (lane w): its scale factors, and whether it holds the
-            // crossing of target = u * S_t in index order (CTA by CTA, then warp by warp)
-            const float ftw = ex2(w0.x - Mt), fdw = ex2(w0.w - Md);
-            const float at = ftw / St, ad = fdw / Sd;
             int sel = 0;
             float base = 0.f, target = u_samp * St;
             if (!bad) {
@@ -839,11 +836,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     }
                 }
             }
-            if (lane < kSW) {
-                float4* m = reinterpret_cast<float4*>(&sh.wmsg[par][lane]);
-                m[0] = make_float4(at, ad, ftw, base);
-                m[1] = make_float4(target, __int_as_float(sel), 0.f, 0.f);
-            }
+            if (lane < kSW)
+                *reinterpret_cast<float4*>(&sh.wmsg[par][lane].target) = make_float4(target, __int_as_float(sel), base, 0.f);
             if (leader && lane == 0) {
                 float* f = sh.fin[n & (kSFinRing - 1)];
                 f[0] = Mt;
@@ -856,7 +850,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.scal_bar[par]));
+                mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.sel_bar[par]));
                 if (leader) *reinterpret_cast<volatile int32_t*>(&sh.n_issued) = n + 1;
             }
             ++n;
@@ -888,11 +882,13 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             // cluster has sent its pass-C sums (they did before publishing their next partials)
             auto finalize = [&](int m) -> int {
                 const int par = m & (kSFinRing - 1);
-                wait_cluster(&sh.c_bar[par], (uint32_t)(m / kSFinRing) & 1u);
-                const float2 c0 = sh.tabC[par][4 * lane], c1 = sh.tabC[par][4 * lane + 1];
-                const float2 c2 = sh.tabC[par][4 * lane + 2], c3 = sh.tabC[par][4 * lane + 3];
+                wait_cta(&sh.c_bar[par], (uint32_t)(m / kSFinRing) & 1u);
+                const float4 c0 = sh.tabC[par][4 * lane], c1 = sh.tabC[par][4 * lane + 1];
+                const float4 c2 = sh.tabC[par][4 * lane + 2], c3 = sh.tabC[par][4 * lane + 3];
                 const float A = warp_sum(((c0.x + c1.x) + c2.x) + c3.x);
                 const float PQ = warp_sum(((c0.y + c1.y) + c2.y) + c3.y);
+                const int tok_all = __reduce_max_sync(0xFFFFFFFFu, max(max(__float_as_int(c0.z), __float_as_int(c1.z)),
+                                                                       max(__float_as_int(c2.z), __float_as_int(c3.z))));
                 int done_b = -1;
                 if (lane == 0) {
                     const PosCtx& c = sh.pc[m & (kSPosRing - 1)];
@@ -903,7 +899,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     const uint32_t fl = __float_as_uint(sh.fin[par][6]);
                     const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL) || !alive;
                     const size_t idt = (size_t)b * K1 + i, idd = (size_t)b * Kmax + i;
-                    int tok = sh.token[par];
+                    int tok = tok_all;
                     if (bad) {
                         atomicOr(p.st.status, ADASD_STATUS_NAN);
                         tok = -1;
