@@ -32,6 +32,7 @@ constexpr int kSThreads = (kSW + 2) * 32;        // 384: leaves 168 registers pe
 constexpr int kSRegIter = 6;                     // iterations whose 2^t values stay in registers
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
 constexpr int kSPosRing = 16;                    // positions the control warp keeps described
+constexpr int kSWorkQ = 16;                      // tail work queue entries per CTA
 constexpr int kSFinRing = 4;                     // positions whose sums may await finalisation
 constexpr uint32_t kSPollSpins = 1u << 24;       // polls of a progress counter before giving up
 
@@ -71,6 +72,8 @@ struct __align__(16) SpecShared {
     int32_t n_issued;                 // leader: positions whose messages have been sent
     int32_t n_final;                  // leader: number of positions of this cluster, -1 until known
     int32_t fin_done;                 // leader: positions finalised so far (written by the tail warp)
+    int32_t wq[kSWorkQ];              // non-leader: sequences whose tail this CTA's tail warp must run (-1: stop)
+    uint32_t wq_head, wq_tail;        // written by the leader's tail warp (remotely) / by this CTA's tail warp
     float td[ADASD_KMAX_LIMIT], tH[ADASD_KMAX_LIMIT];   // tail warp scratch
 };
 
@@ -91,6 +94,16 @@ __device__ __forceinline__ void st_async_v4(uint32_t remote_addr, float4 v, uint
                  ::"r"(remote_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(remote_bar)
                  : "memory");
 }
+
+__device__ __forceinline__ void st_cluster_u32(uint32_t remote_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_cluster_u32(uint32_t remote_addr) {
+    uint32_t v;
+    asm volatile("ld.volatile.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(remote_addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 
 // The per-sequence tail of a round, run by ONE warp: lane i owns candidate i.  Same
 // arithmetic as verify_tail (KDE sums over L_D^A and L_D^R, Bayes posterior with the
@@ -246,6 +259,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         sh.n_issued = 0;
         sh.n_final = -1;
         sh.fin_done = 0;
+        sh.wq_head = sh.wq_tail = 0u;
         for (int k = 0; k < 2; ++k) {
             mbar_init(reinterpret_cast<uint64_t*>(&sh.entry_bar[k]), kSW);
             mbar_init(reinterpret_cast<uint64_t*>(&sh.ctab_bar[k]), 1);
@@ -941,6 +955,33 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 return __shfl_sync(0xFFFFFFFFu, done_b, 0);
             };
 
+            // tails go round robin to the tail warps of the other CTAs of the cluster, which have
+            // nothing else to do: entry number k of CTA r's queue
+            uint32_t ndisp = 0;
+            auto send = [&](uint32_t r, uint32_t k, int b) {
+                if (lane == 0) {
+                    const uint32_t tail_addr = mapa_u32(&sh.wq_tail, r);
+                    bool room = !alive;
+                    for (uint32_t it = 0; !room && it < kSPollSpins; ++it) {
+                        room = (k - ld_cluster_u32(tail_addr)) < (uint32_t)kSWorkQ;
+                        if (!room) __nanosleep(100);
+                    }
+                    if (room) {
+                        __threadfence();
+                        st_cluster_u32(mapa_u32(&sh.wq[k % kSWorkQ], r), (uint32_t)b);
+                        fence_cluster();
+                        st_cluster_u32(mapa_u32(&sh.wq_head, r), k + 1u);
+                    } else {
+                        atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                    }
+                }
+                __syncwarp();
+            };
+            auto dispatch = [&](int b) {
+                const uint32_t nw = (uint32_t)(CS - 1);
+                send(1u + ndisp % nw, ndisp / nw, b);
+                ++ndisp;
+            };
             for (int m = 0;; ++m) {
                 // position m exists once its messages have gone out; the control warp says when
                 // the cluster has no more
@@ -963,13 +1004,58 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 if (go <= 0) break;
                 const int done_b = finalize(m);
                 if (done_b >= 0) {
-                    __threadfence();
-                    verify_tail_warp(p.tail, io, p.st, done_b, sh.td, sh.tH);
+                    if (CS > 1) {
+                        dispatch(done_b);
+                    } else {
+                        __threadfence();
+                        verify_tail_warp(p.tail, io, p.st, done_b, sh.td, sh.tH);
+                    }
                 }
                 if (lane == 0) {
                     __threadfence_block();
                     *reinterpret_cast<volatile int32_t*>(&sh.fin_done) = m + 1;
                 }
+            }
+            // stop marks: CTA r has received the entries ndisp' < ndisp with ndisp' % nw == r - 1
+            for (uint32_t r = 1; r < (uint32_t)CS; ++r) {
+                const uint32_t nw = (uint32_t)(CS - 1);
+                const uint32_t sent = ndisp / nw + ((ndisp % nw) > (r - 1u) ? 1u : 0u);
+                send(r, sent, -1);
+            }
+        } else {
+            // worker: tails handed over by the leader's tail warp, in order, until the stop mark
+            TailIO io;
+            io.H_d = p.sc.H_d;
+            io.dist = p.sc.dist;
+            io.y = p.sc.y;
+            io.x = p.x;
+            io.u_accept = p.u_accept;
+            io.draft_len = p.draft_len;
+            io.p_acc = p.sc.p_acc;
+            io.p_acc_user = p.user.p_acc;
+            io.accept_len = p.accept_len;
+            io.next_token = p.next_token;
+            io.accept_len_rec = p.user.accept_len;
+            io.rejected_rec = p.user.rejected;
+            io.draft_len_rec = p.user.draft_len;
+            for (uint32_t k = 0;; ++k) {
+                int b = -2;
+                if (lane == 0) {
+                    for (uint32_t it = 0; it < kSPollSpins; ++it) {
+                        if (*reinterpret_cast<volatile uint32_t*>(&sh.wq_head) != k) {
+                            fence_cluster();
+                            b = *reinterpret_cast<volatile int32_t*>(&sh.wq[k % kSWorkQ]);
+                            break;
+                        }
+                        __nanosleep(200);
+                    }
+                    if (b == -2) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                }
+                b = __shfl_sync(0xFFFFFFFFu, b, 0);
+                if (b < 0) break;            // stop mark, or nothing ever came
+                __threadfence();
+                verify_tail_warp(p.tail, io, p.st, b, sh.td, sh.tH);
+                if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&sh.wq_tail) = k + 1u;
             }
         }
     }
