@@ -481,67 +481,81 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const float2 L2 = make_float2(kLog2e, kLog2e);
             const float2 nmt = make_float2(nmt_w, nmt_w);
             const float2 nmd = make_float2(nmd_w, nmd_w);
+            // The logits of iteration k + 1 are fetched from the ring before iteration k is worked
+            // on, so neither the shared-memory latency nor the refill at a slot's end (which the
+            // compiler may not move loads across) leaves the SFU pipe without work.
+            uint4 Tn = make_uint4(0u, 0u, 0u, 0u), Dn = Tn;
+            auto fetch = [&](int k, int slot) {
+                const unsigned char* sb = ring + (size_t)slot * kCSlotBytes + (size_t)lane * 16 + (k & 1) * 512;
+                Tn = *reinterpret_cast<const uint4*>(sb);
+                mask_unit(k, Tn);
+                if (!BONUS) {
+                    Dn = *reinterpret_cast<const uint4*>(sb + 1024);
+                    mask_unit(k, Dn);
+                }
+            };
+            if (k_on(0)) fetch(0, cons_slot);
 #pragma unroll
-            for (int st = 0; st < NSTG; ++st) {
-                if ((2 * st < ITER - 1) || full) {                       // the stage exists for this warp
-                    const unsigned char* sb = ring + (size_t)cons_slot * kCSlotBytes + (size_t)lane * 16;
+            for (int k = 0; k < ITER; ++k) {
+                if (k_on(k)) {
+                    const uint4 T = Tn, D = Dn;
+                    if (k + 1 < ITER && k_on(k + 1)) {
+                        int slot = cons_slot;
+                        if (k & 1) {                       // iteration k + 1 opens the next slot
+                            if (++slot == NSw) slot = 0;
+                        }
+                        fetch(k + 1, slot);
+                    }
+                    float e1[8], e2[8];
+                    const uint32_t tw[4] = {T.x, T.y, T.z, T.w};
 #pragma unroll
-                    for (int kk = 0; kk < 2; ++kk) {
-                        const int k = 2 * st + kk;
-                        if (k < ITER && k_on(k)) {
-                            float e1[8], e2[8];
-                            uint4 T = *reinterpret_cast<const uint4*>(sb + kk * 512);
-                            mask_unit(k, T);
-                            const uint32_t tw[4] = {T.x, T.y, T.z, T.w};
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 z = unpack2(bclamp2(tw[j]));
+                        const float2 t = __ffma2_rn(z, L2, nmt);
+                        const float2 e = make_float2(ex2(t.x), ex2(t.y));
+                        e1[2 * j] = e.x;
+                        e1[2 * j + 1] = e.y;
+                        St = __fadd2_rn(St, e);
+                        Tt = __ffma2_rn(e, t, Tt);
+                    }
+                    if (!BONUS) {
+                        const uint32_t dw[4] = {D.x, D.y, D.z, D.w};
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float2 z = unpack2(bclamp2(tw[j]));
-                                const float2 t = __ffma2_rn(z, L2, nmt);
-                                const float2 e = make_float2(ex2(t.x), ex2(t.y));
-                                e1[2 * j] = e.x;
-                                e1[2 * j + 1] = e.y;
-                                St = __fadd2_rn(St, e);
-                                Tt = __ffma2_rn(e, t, Tt);
-                            }
-                            if (!BONUS) {
-                                uint4 D = *reinterpret_cast<const uint4*>(sb + 1024 + kk * 512);
-                                mask_unit(k, D);
-                                const uint32_t dw[4] = {D.x, D.y, D.z, D.w};
+                        for (int j = 0; j < 4; ++j) {
+                            const float2 z = unpack2(bclamp2(dw[j]));
+                            const float2 t = __ffma2_rn(z, L2, nmd);
+                            const float2 e = make_float2(ex2(t.x), ex2(t.y));
+                            e2[2 * j] = e.x;
+                            e2[2 * j + 1] = e.y;
+                            Sd = __fadd2_rn(Sd, e);
+                            Td = __ffma2_rn(e, t, Td);
+                        }
+                    } else {
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    const float2 z = unpack2(bclamp2(dw[j]));
-                                    const float2 t = __ffma2_rn(z, L2, nmd);
-                                    const float2 e = make_float2(ex2(t.x), ex2(t.y));
-                                    e2[2 * j] = e.x;
-                                    e2[2 * j + 1] = e.y;
-                                    Sd = __fadd2_rn(Sd, e);
-                                    Td = __ffma2_rn(e, t, Td);
-                                }
-                            } else {
+                        for (int j = 0; j < 8; ++j) e2[j] = 0.f;
+                    }
+                    if (k < KR) {
 #pragma unroll
-                                for (int j = 0; j < 8; ++j) e2[j] = 0.f;
-                            }
-                            if (k < KR) {
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    et[k < KR ? k : 0][j] = e1[j];
-                                    ed[k < KR ? k : 0][j] = e2[j];
-                                }
-                            } else {
-                                *stash_ptr(k, 0) = make_float4(e1[0], e1[1], e1[2], e1[3]);
-                                *stash_ptr(k, 1) = make_float4(e1[4], e1[5], e1[6], e1[7]);
-                                if (!BONUS) {
-                                    *stash_ptr(k, 2) = make_float4(e2[0], e2[1], e2[2], e2[3]);
-                                    *stash_ptr(k, 3) = make_float4(e2[4], e2[5], e2[6], e2[7]);
-                                }
-                            }
+                        for (int j = 0; j < 8; ++j) {
+                            et[k < KR ? k : 0][j] = e1[j];
+                            ed[k < KR ? k : 0][j] = e2[j];
+                        }
+                    } else {
+                        *stash_ptr(k, 0) = make_float4(e1[0], e1[1], e1[2], e1[3]);
+                        *stash_ptr(k, 1) = make_float4(e1[4], e1[5], e1[6], e1[7]);
+                        if (!BONUS) {
+                            *stash_ptr(k, 2) = make_float4(e2[0], e2[1], e2[2], e2[3]);
+                            *stash_ptr(k, 3) = make_float4(e2[4], e2[5], e2[6], e2[7]);
                         }
                     }
-                    // the slot is consumed: flip its parity and refill it with the next stage
-                    __syncwarp();
-                    phase ^= 1u << cons_slot;
-                    issue_one(cons_slot);
-                    if (++cons_slot == NSw) cons_slot = 0;
+                    if ((k & 1) || k == ITER - 1 || !k_on(k + 1)) {
+                        // the slot is consumed (both its iterations are in registers or done): flip
+                        // its parity and refill it with the next stage
+                        __syncwarp();
+                        phase ^= 1u << cons_slot;
+                        issue_one(cons_slot);
+                        if (++cons_slot == NSw) cons_slot = 0;
+                    }
                 }
             }
             sB[0] = warp_sum(St.x + St.y);
