@@ -185,17 +185,27 @@ void fast_setup_mode(adasd_ctx* c, size_t smem_optin) {
         const int ncu = (NU + cs - 1) / cs, nwi = (ncu + 31) / 32;
         const int I_lo = nwi / warps, rem = nwi % warps, iter = I_lo + (rem ? 1 : 0);
         if (iter < 1 || iter > kCMaxIter) continue;
-        const int KR = std::min(iter, reg_iter);
-        int stash_slots = 0;
-        if (iter > KR) stash_slots = (iter - 1 - KR) * warps + ((iter - 1 < I_lo) ? warps : rem);
-        const int stash_bytes = stash_slots * kCSlotBytes;
         const int st = fast_static_smem_iter<MODE>(iter);
         if (st < 0) continue;
-        const int avail = (int)smem_optin - st - stash_bytes - 1024;
-        const int n_stg = (iter + 1) / 2;
-        int NS = std::min({kCMaxSlots, avail / (warps * kCSlotBytes), 2 * n_stg});
-        if (NS < n_stg) continue;
-        const int smem = NS * warps * kCSlotBytes + stash_bytes;
+        int NS, smem, stash_off;
+        if (MODE == MODE_ADASD) {
+            // two position buffers per compute warp, iter * 512 bytes per row; nothing else
+            NS = 2;
+            smem = warps * iter * 2048;
+            stash_off = 0;
+            if (smem > (int)smem_optin - st - 1024) continue;
+        } else {
+            const int KR = std::min(iter, reg_iter);
+            int stash_slots = 0;
+            if (iter > KR) stash_slots = (iter - 1 - KR) * warps + ((iter - 1 < I_lo) ? warps : rem);
+            const int stash_bytes = stash_slots * kCSlotBytes;
+            const int avail = (int)smem_optin - st - stash_bytes - 1024;
+            const int n_stg = (iter + 1) / 2;
+            NS = std::min({kCMaxSlots, avail / (warps * kCSlotBytes), 2 * n_stg});
+            if (NS < n_stg) continue;
+            smem = NS * warps * kCSlotBytes + stash_bytes;
+            stash_off = NS * warps * kCSlotBytes;
+        }
         const int ncl = fast_occupancy_iter<MODE>(iter, cs, smem);
         const int score = ncl * cs;
         if (score > best_score) {
@@ -204,7 +214,7 @@ void fast_setup_mode(adasd_ctx* c, size_t smem_optin) {
             f.cs = cs;
             f.smem = smem;
             f.geom.NS = NS;
-            f.geom.stash_off = NS * warps * kCSlotBytes;
+            f.geom.stash_off = stash_off;
             f.geom.ncl = ncl;
         }
     }

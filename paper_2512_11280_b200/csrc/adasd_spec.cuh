@@ -68,7 +68,7 @@ struct __align__(16) SpecShared {
     unsigned long long scal_bar[2];   // 1 arrival: first part of wmsg[par] ready
     unsigned long long sel_bar[2];    // 1 arrival: second part of wmsg[par] ready
     unsigned long long c_bar[kSFinRing];   // leader: 16 bytes from every compute warp of the cluster: tabC complete
-    unsigned long long bar[kCW][kCMaxSlots];   // "slot filled" barriers
+    unsigned long long bar[kCW][2];   // per compute warp: "position buffer filled" barriers
     int32_t n_issued;                 // leader: positions whose messages have been sent
     int32_t n_final;                  // leader: number of positions of this cluster, -1 until known
     int32_t fin_done;                 // leader: positions finalised so far (written by the tail warp)
@@ -232,7 +232,6 @@ template <int ITER>
 __global__ void __launch_bounds__(kSThreads, 1)
 spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
     constexpr int KR = ITER < kSRegIter ? ITER : kSRegIter;   // iterations kept in registers
-    constexpr int NSTG = (ITER + 1) / 2;                      // slots of one position, at most
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ SpecShared sh;
 
@@ -269,7 +268,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         for (int k = 0; k < kSFinRing; ++k) mbar_init(reinterpret_cast<uint64_t*>(&sh.c_bar[k]), 1);
     }
     if (warp < kSW && lane == 0)
-        for (int s = 0; s < kCMaxSlots; ++s) mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][s]), 1);
+        for (int s = 0; s < 2; ++s) mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][s]), 1);
     __syncthreads();
 
     // first active position among start, start + ncl, ... (32 candidates per round)
@@ -356,44 +355,33 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         const int wi0 = warp * I_lo + min(warp, I_rem);
         const int wu0 = cu0 + 32 * wi0;
         const int nwu = max(0, min(32 * I_w, cu1 - wu0));          // units of this warp (last one ragged)
-        const int n_stg = (I_w + 1) >> 1;                          // ring slots one position takes
-        const int NSw = min(gq.NS, 2 * n_stg);                     // slots this warp cycles through
-        const uint32_t last_bytes = n_stg > 0 ? (uint32_t)(nwu - 64 * (n_stg - 1)) * 16u : 0u;
-        const size_t woff = (size_t)wi0 * 512;                     // byte offset of the share in the CTA's slice
+        const uint32_t row_bytes = (uint32_t)nwu * 16u;            // this warp's share of one row
+        const size_t woff = (size_t)wi0 * 512;                     // its byte offset in the CTA's slice
 
-        unsigned char* const ring = dyn_smem + (size_t)warp * gq.NS * kCSlotBytes;
-        unsigned char* const stash = dyn_smem + gq.stash_off + (size_t)warp * kCSlotBytes + (size_t)lane * 16;
-        auto stash_ptr = [&](int k, int plane) -> float4* {
-            return reinterpret_cast<float4*>(stash + (size_t)(k - KR) * (kSW * kCSlotBytes) + plane * 512);
-        };
+        // Two buffers per warp, one position each: [target share | draft share], ITER * 512 bytes
+        // per row.  Position n lives in buffer n & 1 and is replaced by position n + 2 as soon as
+        // pass C of position n is done, one whole position before it is needed.
+        constexpr int kRowB = ITER * 512;
+        unsigned char* const bufs = dyn_smem + (size_t)warp * (4 * kRowB);
+        auto buf_of = [&](int n) -> unsigned char* { return bufs + (size_t)(n & 1) * (2 * kRowB) + (size_t)lane * 16; };
+        auto bar_of = [&](int n) -> uint64_t* { return reinterpret_cast<uint64_t*>(&sh.bar[warp][n & 1]); };
         auto pcx = [&](int n) -> const PosCtx& { return sh.pc[n & (kSPosRing - 1)]; };
 
-        int n = 0;                 // sequence number of the current position
-        uint32_t phase = 0;        // bit s: parity to wait for on slot s
-        int cons_slot = 0;         // slot holding the next stage to be consumed
-        int ip_which = 0;          // position the next fill belongs to: n + ip_which (at most n + 2)
-        int ip_stage = 0;          // its next stage
-        auto bar_of = [&](int s) -> uint64_t* { return reinterpret_cast<uint64_t*>(&sh.bar[warp][s]); };
-        auto issue_one = [&](int slot) {
-            if (!alive || n_stg == 0 || ip_which > 2) return;
-            const PosCtx& c = pcx(n + ip_which);
-            if (c.pos >= total) return;
-            if (lane == 0) {
-                const uint32_t bytes = (ip_stage == n_stg - 1) ? last_bytes : 1024u;
-                const bool bonus = c.bonus != 0;
-                unsigned char* dst = ring + (size_t)slot * kCSlotBytes;
-                uint64_t* bar = bar_of(slot);
-                const size_t off = woff + (size_t)ip_stage * 1024;
-                mbar_expect_tx(bar, bonus ? bytes : 2u * bytes);
-                bulk_g2s(dst, reinterpret_cast<const unsigned char*>(c.src_t) + off, bytes, bar);
-                if (!bonus) bulk_g2s(dst + 1024, reinterpret_cast<const unsigned char*>(c.src_d) + off, bytes, bar);
-            }
-            if (++ip_stage == n_stg) {
-                ip_stage = 0;
-                ++ip_which;
-            }
+        // lanes 0 and 1 fetch the two rows of position n (lane 1 idles for a bonus row)
+        auto issue_pos = [&](int n) {
+            const PosCtx& c = pcx(n);
+            if (!alive || nwu == 0 || c.pos >= total) return;
+            const bool bonus = c.bonus != 0;
+            uint64_t* bar = bar_of(n);
+            unsigned char* dst = bufs + (size_t)(n & 1) * (2 * kRowB);
+            if (lane == 0) mbar_expect_tx(bar, bonus ? row_bytes : 2u * row_bytes);
+            __syncwarp();
+            if (lane < (bonus ? 1 : 2))
+                bulk_g2s(dst + lane * kRowB,
+                         reinterpret_cast<const unsigned char*>(lane ? c.src_d : c.src_t) + woff, row_bytes, bar);
         };
-        for (int s = 0; s < NSw; ++s) issue_one(s);
+        issue_pos(0);
+        issue_pos(1);
 
         // iteration k runs for this warp: all but the last always do
         auto k_on = [&](int k) -> bool { return (k < ITER - 1) || full; };
@@ -404,48 +392,42 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 w = make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
         };
 
-        // ---- pass A: packed maxima and flags of one position, slot by slot ------------------
+        // ---- pass A: packed maxima and flags of one position ---------------------------------
         uint32_t a_mT = 0xFF80FF80u, a_mD = 0xFF80FF80u, a_df = 0u;   // -inf pairs
-        int a_next = 0;                                                 // first stage not yet scanned
-        auto pass_a = [&](auto bonus_c, bool blocking) {
+        bool a_done = false;
+        // with blocking == false it gives up at once if the position has not landed yet
+        auto pass_a = [&](auto bonus_c, int n, bool blocking) {
             constexpr bool BONUS = decltype(bonus_c)::value;
-            if (!alive) return;
+            if (!alive || a_done) return;
+            if (nwu > 0) {
+                const uint32_t par = (uint32_t)(n >> 1) & 1u;
+                bool ok = blocking ? mbar_wait_bounded(bar_of(n), par) : (mbar_test_wait(bar_of(n), par) != 0);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) {
+                    if (blocking) expired();     // the copy never landed
+                    return;
+                }
+            }
+            a_done = true;
+            const unsigned char* sb = buf_of(n);
 #pragma unroll
-            for (int st = 0; st < NSTG; ++st) {
-                if (st >= a_next && st < n_stg) {
-                    int slot = cons_slot + st;
-                    if (slot >= NSw) slot -= NSw;
-                    const uint32_t par = (phase >> slot) & 1u;
-                    bool ok = blocking ? mbar_wait_bounded(bar_of(slot), par)
-                                       : (mbar_test_wait(bar_of(slot), par) != 0);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) {
-                        if (blocking) expired();     // the copy never landed
-                        break;
-                    }
-                    a_next = st + 1;
-                    const unsigned char* sb = ring + (size_t)slot * kCSlotBytes + (size_t)lane * 16;
-#pragma unroll
-                    for (int kk = 0; kk < 2; ++kk) {
-                        const int k = 2 * st + kk;
-                        if (k < ITER && k_on(k)) {
-                            uint4 T = *reinterpret_cast<const uint4*>(sb + kk * 512);
-                            mask_unit(k, T);
-                            a_mT = bmax2(bmax2(a_mT, T.x), bmax2(T.y, bmax2(T.z, T.w)));
-                            if (!BONUS) {
-                                uint4 D = *reinterpret_cast<const uint4*>(sb + 1024 + kk * 512);
-                                mask_unit(k, D);
-                                a_mD = bmax2(bmax2(a_mD, D.x), bmax2(D.y, bmax2(D.z, D.w)));
-                                a_df |= (T.x ^ D.x) | (T.y ^ D.y) | (T.z ^ D.z) | (T.w ^ D.w);
-                            }
-                        }
+            for (int k = 0; k < ITER; ++k) {
+                if (k_on(k)) {
+                    uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
+                    mask_unit(k, T);
+                    a_mT = bmax2(bmax2(a_mT, T.x), bmax2(T.y, bmax2(T.z, T.w)));
+                    if (!BONUS) {
+                        uint4 D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
+                        mask_unit(k, D);
+                        a_mD = bmax2(bmax2(a_mD, D.x), bmax2(D.y, bmax2(D.z, D.w)));
+                        a_df |= (T.x ^ D.x) | (T.y ^ D.y) | (T.z ^ D.z) | (T.w ^ D.w);
                     }
                 }
             }
         };
-        auto pass_a_any = [&](bool bonus, bool blocking) {
-            if (bonus) pass_a(std::true_type{}, blocking);
-            else pass_a(std::false_type{}, blocking);
+        auto pass_a_any = [&](bool bonus, int n, bool blocking) {
+            if (bonus) pass_a(std::true_type{}, n, blocking);
+            else pass_a(std::false_type{}, n, blocking);
         };
 
         // The warp's shifts and flags from the packed accumulators.  Shifts live in the log2
@@ -469,67 +451,44 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             flags_w = __reduce_or_sync(0xFFFFFFFFu, bad | (a_df ? 2u : 0u));
             a_mT = a_mD = 0xFF80FF80u;
             a_df = 0u;
-            a_next = 0;
+            a_done = false;
         };
 
-        // ---- pass B: 2^t values (kept) and the warp's S and T --------------------------------
+        // 2^t values of one unit: 8 logits (four packed words) relative to the shift in `nm`
+        auto exps = [&](const uint4& W, const float2 nm, float (&e)[8], float2& S, float2& Tq) {
+            const float2 L2 = make_float2(kLog2e, kLog2e);
+            const uint32_t w[4] = {W.x, W.y, W.z, W.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 z = unpack2(bclamp2(w[j]));
+                const float2 t = __ffma2_rn(z, L2, nm);
+                const float2 v = make_float2(ex2(t.x), ex2(t.y));
+                e[2 * j] = v.x;
+                e[2 * j + 1] = v.y;
+                S = __fadd2_rn(S, v);
+                Tq = __ffma2_rn(v, t, Tq);
+            }
+        };
+
+        // ---- pass B: the warp's S and T; the 2^t values of the first KR iterations are kept ----
         float et[KR][8], ed[KR][8];
         float sB[4];                       // after pass_b: warp totals St, Tt, Sd, Td
-        auto pass_b = [&](auto bonus_c) {
+        auto pass_b = [&](auto bonus_c, int n) {
             constexpr bool BONUS = decltype(bonus_c)::value;
             float2 St = make_float2(0.f, 0.f), Tt = St, Sd = St, Td = St;
-            const float2 L2 = make_float2(kLog2e, kLog2e);
-            const float2 nmt = make_float2(nmt_w, nmt_w);
-            const float2 nmd = make_float2(nmd_w, nmd_w);
-            // The logits of iteration k + 1 are fetched from the ring before iteration k is worked
-            // on, so neither the shared-memory latency nor the refill at a slot's end (which the
-            // compiler may not move loads across) leaves the SFU pipe without work.
-            uint4 Tn = make_uint4(0u, 0u, 0u, 0u), Dn = Tn;
-            auto fetch = [&](int k, int slot) {
-                const unsigned char* sb = ring + (size_t)slot * kCSlotBytes + (size_t)lane * 16 + (k & 1) * 512;
-                Tn = *reinterpret_cast<const uint4*>(sb);
-                mask_unit(k, Tn);
-                if (!BONUS) {
-                    Dn = *reinterpret_cast<const uint4*>(sb + 1024);
-                    mask_unit(k, Dn);
-                }
-            };
-            if (k_on(0)) fetch(0, cons_slot);
+            const float2 nmt = make_float2(nmt_w, nmt_w), nmd = make_float2(nmd_w, nmd_w);
+            const unsigned char* sb = buf_of(n);
 #pragma unroll
             for (int k = 0; k < ITER; ++k) {
                 if (k_on(k)) {
-                    const uint4 T = Tn, D = Dn;
-                    if (k + 1 < ITER && k_on(k + 1)) {
-                        int slot = cons_slot;
-                        if (k & 1) {                       // iteration k + 1 opens the next slot
-                            if (++slot == NSw) slot = 0;
-                        }
-                        fetch(k + 1, slot);
-                    }
                     float e1[8], e2[8];
-                    const uint32_t tw[4] = {T.x, T.y, T.z, T.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float2 z = unpack2(bclamp2(tw[j]));
-                        const float2 t = __ffma2_rn(z, L2, nmt);
-                        const float2 e = make_float2(ex2(t.x), ex2(t.y));
-                        e1[2 * j] = e.x;
-                        e1[2 * j + 1] = e.y;
-                        St = __fadd2_rn(St, e);
-                        Tt = __ffma2_rn(e, t, Tt);
-                    }
+                    uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
+                    mask_unit(k, T);
+                    exps(T, nmt, e1, St, Tt);
                     if (!BONUS) {
-                        const uint32_t dw[4] = {D.x, D.y, D.z, D.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float2 z = unpack2(bclamp2(dw[j]));
-                            const float2 t = __ffma2_rn(z, L2, nmd);
-                            const float2 e = make_float2(ex2(t.x), ex2(t.y));
-                            e2[2 * j] = e.x;
-                            e2[2 * j + 1] = e.y;
-                            Sd = __fadd2_rn(Sd, e);
-                            Td = __ffma2_rn(e, t, Td);
-                        }
+                        uint4 D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
+                        mask_unit(k, D);
+                        exps(D, nmd, e2, Sd, Td);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 8; ++j) e2[j] = 0.f;
@@ -540,21 +499,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                             et[k < KR ? k : 0][j] = e1[j];
                             ed[k < KR ? k : 0][j] = e2[j];
                         }
-                    } else {
-                        *stash_ptr(k, 0) = make_float4(e1[0], e1[1], e1[2], e1[3]);
-                        *stash_ptr(k, 1) = make_float4(e1[4], e1[5], e1[6], e1[7]);
-                        if (!BONUS) {
-                            *stash_ptr(k, 2) = make_float4(e2[0], e2[1], e2[2], e2[3]);
-                            *stash_ptr(k, 3) = make_float4(e2[4], e2[5], e2[6], e2[7]);
-                        }
-                    }
-                    if ((k & 1) || k == ITER - 1 || !k_on(k + 1)) {
-                        // the slot is consumed (both its iterations are in registers or done): flip
-                        // its parity and refill it with the next stage
-                        __syncwarp();
-                        phase ^= 1u << cons_slot;
-                        issue_one(cons_slot);
-                        if (++cons_slot == NSw) cons_slot = 0;
                     }
                 }
             }
@@ -568,8 +512,10 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 sB[3] = warp_sum(Td.x + Td.y);
             }
         };
-        // the 2^t values of iteration k (compile-time k after unrolling)
-        auto load_stash = [&](int k, float (&a)[8], float (&b)[8]) {
+        // The 2^t values of iteration k (compile-time k after unrolling): kept ones from
+        // registers, the others worked out again from the logits, which stay in the buffer until
+        // pass C is over (ex2 is cheap; shared-memory bandwidth for a second copy is not).
+        auto load_kept = [&](int k, int n, bool with_d, float (&a)[8], float (&b)[8]) {
             if (k < KR) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -577,32 +523,33 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     b[j] = ed[k < KR ? k : 0][j];
                 }
             } else {
-                const float4 a0 = *stash_ptr(k, 0), a1 = *stash_ptr(k, 1), b0 = *stash_ptr(k, 2), b1 = *stash_ptr(k, 3);
-                a[0] = a0.x, a[1] = a0.y, a[2] = a0.z, a[3] = a0.w, a[4] = a1.x, a[5] = a1.y, a[6] = a1.z, a[7] = a1.w;
-                b[0] = b0.x, b[1] = b0.y, b[2] = b0.z, b[3] = b0.w, b[4] = b1.x, b[5] = b1.y, b[6] = b1.z, b[7] = b1.w;
-            }
-        };
-        auto load_stash_t = [&](int k, float (&a)[8]) {      // target values only
-            if (k < KR) {
+                const unsigned char* sb = buf_of(n);
+                float2 s0 = make_float2(0.f, 0.f), s1 = s0;
+                uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
+                mask_unit(k, T);
+                exps(T, make_float2(nmt_w, nmt_w), a, s0, s1);
+                if (with_d) {
+                    uint4 D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
+                    mask_unit(k, D);
+                    exps(D, make_float2(nmd_w, nmd_w), b, s0, s1);
+                } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) a[j] = et[k < KR ? k : 0][j];
-            } else {
-                const float4 a0 = *stash_ptr(k, 0), a1 = *stash_ptr(k, 1);
-                a[0] = a0.x, a[1] = a0.y, a[2] = a0.z, a[3] = a0.w, a[4] = a1.x, a[5] = a1.y, a[6] = a1.z, a[7] = a1.w;
+                    for (int j = 0; j < 8; ++j) b[j] = 0.f;
+                }
             }
         };
 
         // Run by the warp that holds the crossing: first element (index order: iteration, lane,
         // element) of the target row where base + f * running weight exceeds target, else the
         // last element with weight.
-        auto select_kept = [&](float base, float f, float target) -> int {
+        auto select_kept = [&](int n, float base, float f, float target) -> int {
             float ls[ITER], tot[ITER];
 #pragma unroll
             for (int k = 0; k < ITER; ++k) {
                 ls[k] = 0.f;
                 if (k_on(k)) {
-                    float v[8];
-                    load_stash_t(k, v);
+                    float v[8], d[8];
+                    load_kept(k, n, false, v, d);
                     ls[k] = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
                 }
             }
@@ -634,7 +581,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
 #pragma unroll
             for (int k = 0; k < ITER; ++k) {
                 if (k == ksel) {          // same for the whole warp
-                    load_stash_t(k, v);
+                    float d[8];
+                    load_kept(k, n, false, v, d);
                     lsum = ls[k];
                 }
             }
@@ -663,7 +611,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         };
 
         // ---------------------------------- main loop ----------------------------------------
-        if (pcx(0).pos < total) pass_a_any(pcx(0).bonus != 0, true);
+        int n = 0;                 // sequence number of the current position
+        if (pcx(0).pos < total) pass_a_any(pcx(0).bonus != 0, 0, true);
         while (pcx(n).pos < total) {
             const int par = n & 1;
             const uint32_t ph = (uint32_t)(n >> 1) & 1u;
@@ -672,8 +621,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const bool nbonus = npos < total && pcx(n + 1).bonus != 0;
 
             finish_a(bonus);
-            if (bonus) pass_b(std::true_type{});
-            else pass_b(std::false_type{});
+            if (bonus) pass_b(std::true_type{}, n);
+            else pass_b(std::false_type{}, n);
             if (lane == 0) {
                 float4* w = reinterpret_cast<float4*>(&sh.wtab[par][warp]);
                 w[0] = make_float4(Mt_w, sB[0], sB[1], Md_w);
@@ -681,9 +630,9 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.entry_bar[par]));
             }
             __syncwarp();
-            // while the control warps exchange the totals: maxima of the next position, as far
-            // as its slots have landed
-            if (npos < total) pass_a_any(nbonus, false);
+            // while the control warps exchange the totals: maxima of the next position, if it
+            // has landed in the other buffer
+            if (npos < total) pass_a_any(nbonus, n + 1, false);
             wait_cta(&sh.scal_bar[par], ph);
             const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft
 
@@ -697,7 +646,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 for (int k = 0; k < ITER; ++k) {
                     if (k_on(k)) {
                         float a[8], d[8];
-                        load_stash(k, a, d);
+                        load_kept(k, n, true, a, d);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const float2 a2 = make_float2(a[2 * j], a[2 * j + 1]);
@@ -718,7 +667,10 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             wait_cta(&sh.sel_bar[par], ph);
             const float4 m1 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp].target); // target, sel, base
             int tok = -1;
-            if (__float_as_int(m1.y) != 0) tok = select_kept(m1.z, m0.z, m1.x);
+            if (__float_as_int(m1.y) != 0) tok = select_kept(n, m1.z, m0.z, m1.x);
+            // the buffer of position n is free: fetch position n + 2 into it
+            __syncwarp();
+            issue_pos(n + 2);
             // this warp's sums (and the token, if it drew it) go to the leader CTA in one message
             if (lane == 0) {
                 const int fr = n & (kSFinRing - 1);
@@ -727,14 +679,15 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             }
             __syncwarp();
 
-            // the rest of the next position's maxima (waits for slots still in flight)
-            if (npos < total) pass_a_any(nbonus, true);
-            --ip_which;
+            // the next position's maxima, if its copy had not landed during the exchange
+            if (npos < total) pass_a_any(nbonus, n + 1, true);
             ++n;
         }
         // a warp that gave up on a copy still waits (bounded) for whatever it had in flight
-        if (!alive)
-            for (int s = 0; s < NSw; ++s) mbar_wait_bounded(bar_of(s), (phase >> s) & 1u);
+        if (!alive && nwu > 0) {
+            mbar_wait_bounded(bar_of(n), (uint32_t)(n >> 1) & 1u);
+            mbar_wait_bounded(bar_of(n + 1), (uint32_t)((n + 1) >> 1) & 1u);
+        }
     } else if (warp == kSCtl) {
         // ============================== control warp ======================================
         auto sum8 = [&](float v) -> float {       // total of the first eight lanes, in every lane
