@@ -13,6 +13,7 @@
 #include "adasd_rows.cuh"
 #include "adasd_cluster.cuh"
 #include "adasd_spec.cuh"
+#include "adasd_draft.cuh"
 
 using namespace adasd;
 
@@ -30,6 +31,7 @@ struct adasd_ctx {
         int smem;             // dynamic shared memory per CTA
         ClusterGeom geom;
     } fast[2];
+    bool draft_stream;        // the streaming draft kernel is usable for this V / dtype
 };
 
 namespace {
@@ -222,6 +224,31 @@ void fast_setup_mode(adasd_ctx* c, size_t smem_optin) {
 void fast_setup(adasd_ctx* c, size_t smem_optin) {
     fast_setup_mode<MODE_ADASD>(c, smem_optin);
     fast_setup_mode<MODE_VANILLA>(c, smem_optin);
+    // streaming draft kernel: bf16 rows of a multiple of 8 logits, two 4 KB buffers per warp
+    c->draft_stream = false;
+    const int V = c->cfg.V;
+    if (c->cfg.dtype == ADASD_BF16 && (V & 7) == 0 && V >= 8192 &&
+        (V >> 3) <= kDMaxP * kDW * kDMaxChunks * kDChunkUnits) {
+        if (cudaFuncSetAttribute(draft_stream_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kDW * 2 * kDChunkBytes) == cudaSuccess)
+            c->draft_stream = true;
+        else
+            cudaGetLastError();
+    }
+}
+
+// CTAs per row for the streaming draft kernel: enough to fill the SMs, and few enough chunks
+// per warp for its tables
+int draft_stream_p(const adasd_ctx* c) {
+    const int NU = c->cfg.V >> 3;
+    int P = 1;
+    if (c->cfg.cluster_size == 1 || c->cfg.cluster_size == 2 || c->cfg.cluster_size == 4 ||
+        c->cfg.cluster_size == 8)
+        P = c->cfg.cluster_size;
+    else
+        while (P < kDMaxP && (long long)c->cfg.B * P * 4 < 3LL * c->sm_count) P *= 2;
+    while (P < kDMaxP && (NU + P * kDW - 1) / (P * kDW) > kDMaxChunks * kDChunkUnits) P *= 2;
+    return P;
 }
 
 template <int ITER, int MODE>
@@ -489,6 +516,24 @@ int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stri
     const int cs = pick_cluster(ctx, p.B);
     const bool vec = vec_ok(logits_dev, ctx->cfg.dtype, {row_stride});
     cudaStream_t st = (cudaStream_t)stream;
+    if (vec && ctx->draft_stream) {
+        const int P = draft_stream_p(ctx);
+        cudaLaunchConfig_t lc;
+        memset(&lc, 0, sizeof(lc));
+        lc.gridDim = dim3((unsigned)(p.B * P), 1, 1);
+        lc.blockDim = dim3(kDThreads, 1, 1);
+        lc.dynamicSmemBytes = (size_t)(kDW * 2 * kDChunkBytes);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)P;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<0>, p));
+        return ADASD_OK;
+    }
     if (ctx->cfg.dtype == ADASD_BF16)
         return vec ? launch_cluster(draft_kernel<__nv_bfloat16, true>, p, p.B, cs, st)
                    : launch_cluster(draft_kernel<__nv_bfloat16, false>, p, p.B, cs, st);

@@ -1,0 +1,240 @@
+// Streaming draft-step kernel for sm_100a (adasd_draft_entropy on bf16 rows of a multiple of 8
+// logits): every row is read from HBM once.
+//
+//  * One cluster of P CTAs per row (P = 1, 2, 4 or 8, chosen so that the launch fills the SMs);
+//    the 8 warps of a CTA split the CTA's part of the row into contiguous shares and stream
+//    them through two 4 KB buffers each (1-D bulk copies, bounded mbarrier waits).
+//  * Per chunk: packed bf16 maximum, then 2^(z log2 e - M) with the warp's running shift M
+//    (raised, with the sums rescaled, only when a chunk exceeds it), accumulating S = sum 2^t
+//    and T = sum 2^t t.  The chunk's own sum is kept in a small table for sampling.
+//  * The CTAs send their totals and tables to rank 0 over DSMEM; after ONE cluster barrier
+//    rank 0 forms H(q) = ln 2 (log2 S - T / S), the log-sum-exp and the stop flag H > T_G,
+//    finds the chunk that holds the inverse-CDF crossing of u and rescans just that chunk
+//    (4 KB, from L2) for the token x ~ q.
+#pragma once
+
+#include "adasd_cluster.cuh"
+
+namespace adasd {
+
+constexpr int kDW = 8;                         // warps per CTA
+constexpr int kDThreads = kDW * 32;
+constexpr int kDChunkUnits = 256;              // 16-byte units per chunk: 8 iterations of a warp
+constexpr int kDChunkBytes = kDChunkUnits * 16;
+constexpr int kDMaxChunks = 12;                // chunks per warp, at most (V <= 8 * 8 * 12 * 2048)
+constexpr int kDMaxP = 8;
+
+struct __align__(16) DraftShared {
+    float cm[kDMaxP][kDW][kDMaxChunks];        // rank 0: shift in force when a chunk was summed
+    float cs[kDMaxP][kDW][kDMaxChunks];        // rank 0: the chunk's sum of 2^t under that shift
+    float4 wpart[kDMaxP][kDW];                 // rank 0: every warp's (M, S, T, flags)
+    unsigned long long bar[kDW][2];
+};
+
+template <int DUMMY = 0>
+__global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams p) {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ DraftShared sh;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int P = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+    const int b = blockIdx.x / P;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool active = !(p.active && p.active[b] == 0);      // same in every CTA of the cluster
+
+    // this warp's share of the row, in 16-byte units
+    const int NU = p.V >> 3;
+    const int cu0 = (int)((long long)rank * NU / P), cu1 = (int)((long long)(rank + 1) * NU / P);
+    const int wu0 = cu0 + (int)((long long)warp * (cu1 - cu0) / kDW);
+    const int wu1 = cu0 + (int)((long long)(warp + 1) * (cu1 - cu0) / kDW);
+    const int nwu = wu1 - wu0;
+    const int nch = min(kDMaxChunks, (nwu + kDChunkUnits - 1) / kDChunkUnits);
+    const unsigned char* const src =
+        reinterpret_cast<const unsigned char*>(reinterpret_cast<const __nv_bfloat16*>(p.z) + (long long)b * p.row_stride) +
+        (size_t)wu0 * 16;
+    unsigned char* const bufs = dyn_smem + (size_t)warp * (2 * kDChunkBytes);
+
+    if (lane == 0) {
+        mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][0]), 1);
+        mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][1]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    cluster.sync();        // every CTA of the cluster is running before anyone writes into rank 0
+    bool alive = true;
+    auto issue = [&](int c) {
+        if (lane == 0 && c < nch) {
+            const uint32_t bytes = (uint32_t)min(kDChunkUnits, nwu - c * kDChunkUnits) * 16u;
+            uint64_t* bar = reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]);
+            mbar_expect_tx(bar, bytes);
+            bulk_g2s(bufs + (size_t)(c & 1) * kDChunkBytes, src + (size_t)c * kDChunkBytes, bytes, bar);
+        }
+    };
+    float M = kFloorL;                                   // running shift (log2 domain)
+    float2 S2 = make_float2(0.f, 0.f), T2 = S2;          // lane partials under M
+    uint32_t bad = 0u;
+    if (active) {
+        issue(0);
+        issue(1);
+        for (int c = 0; c < nch; ++c) {
+            bool ok = alive && mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) {
+                if (alive && lane == 0) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                alive = false;
+                bad = 1u;
+                break;
+            }
+            const unsigned char* sb = bufs + (size_t)(c & 1) * kDChunkBytes + (size_t)lane * 16;
+            const int ubase = c * kDChunkUnits + lane;
+            uint4 W[8];
+            uint32_t mx = 0xFF80FF80u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                W[i] = *reinterpret_cast<const uint4*>(sb + i * 512);
+                if (!(ubase + 32 * i < nwu)) W[i] = make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
+                mx = bmax2(bmax2(mx, W[i].x), bmax2(W[i].y, bmax2(W[i].z, W[i].w)));
+            }
+            // both buffers are in registers or free: fetch the chunk after the next
+            __syncwarp();
+            issue(c + 2);
+            const float2 mm = unpack2(mx);
+            if (mm.x != mm.x || mm.y != mm.y) bad = 1u;
+            const float vmax = warp_max_f32(fmaxf(mm.x, mm.y));
+            if (vmax == INFINITY) bad = 1u;
+            const float Mc = vmax > ADASD_FLOOR_BF ? vmax * kLog2e : kFloorL;
+            if (Mc > M) {                                 // raise the shift, rescale what is summed
+                const float d = M - Mc, f = ex2(d);
+                T2.x = f * fmaf(d, S2.x, T2.x);
+                T2.y = f * fmaf(d, S2.y, T2.y);
+                S2.x *= f;
+                S2.y *= f;
+                M = Mc;
+            }
+            const float nm = M > kFloorL ? -M : 0.f;
+            const float2 nm2 = make_float2(nm, nm), L2 = make_float2(kLog2e, kLog2e);
+            float2 Sc = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t w[4] = {W[i].x, W[i].y, W[i].z, W[i].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 z = unpack2(bclamp2(w[j]));
+                    const float2 t = __ffma2_rn(z, L2, nm2);
+                    const float2 e = make_float2(ex2(t.x), ex2(t.y));
+                    Sc = __fadd2_rn(Sc, e);
+                    T2 = __ffma2_rn(e, t, T2);
+                }
+            }
+            S2 = __fadd2_rn(S2, Sc);
+            const float cs = warp_sum(Sc.x + Sc.y);
+            if (lane == 0) {
+                DraftShared* r0 = cluster.map_shared_rank(&sh, 0);
+                r0->cm[rank][warp][c] = M;
+                r0->cs[rank][warp][c] = cs;
+            }
+        }
+        const float Sw = warp_sum(S2.x + S2.y), Tw = warp_sum(T2.x + T2.y);
+        bad = __reduce_or_sync(0xFFFFFFFFu, bad);
+        if (lane == 0)
+            cluster.map_shared_rank(&sh, 0)->wpart[rank][warp] = make_float4(M, Sw, Tw, __uint_as_float(bad));
+    }
+    cluster.sync();        // totals and tables of every CTA are in rank 0's shared memory
+    if (!active || rank != 0) return;
+    // (rank 0 only reads its own shared memory from here on; nobody writes to it any more)
+
+    if (warp == 0) {
+        // row totals: lane l holds warp-entry l (and l + 32 when P * 8 > 32)
+        const int NE = P * kDW;
+        const float4* wp = &sh.wpart[0][0];
+        float4 e0 = lane < NE ? wp[lane] : make_float4(kFloorL, 0.f, 0.f, 0.f);
+        float4 e1 = lane + 32 < NE ? wp[lane + 32] : make_float4(kFloorL, 0.f, 0.f, 0.f);
+        const float Mr = warp_max_f32(fmaxf(e0.x, e1.x));
+        const float d0 = e0.x - Mr, d1 = e1.x - Mr;
+        const float f0 = ex2(d0), f1 = ex2(d1);
+        const float S = warp_sum(f0 * e0.y + f1 * e1.y);
+        const float T = warp_sum(f0 * fmaf(d0, e0.y, e0.z) + f1 * fmaf(d1, e1.y, e1.z));
+        const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(e0.w) | __float_as_uint(e1.w));
+        const bool rowbad = (fl & 1u) || !(Mr > kFloorL);
+        const float lS = lg2(S);
+        float H = kLn2 * (lS - T / S), lse = kLn2 * (Mr + lS);
+        if (rowbad) H = lse = NAN;
+
+        // x ~ q: which chunk holds the crossing of u * S, in index order (rank, warp, chunk)
+        int tok = -1;
+        const bool sampling = (p.u != nullptr && p.token_out != nullptr);
+        if (sampling && !rowbad) {
+            float target = __ldg(p.u + b) * S;
+            const int E = NE * kDMaxChunks;
+            float run = 0.f, base = 0.f, lbase = 0.f;
+            int hit = -1, last = -1;
+            for (int e = 0; e < E && hit < 0; e += 32) {
+                const int idx = e + lane;
+                const int r = idx / (kDW * kDMaxChunks), w = (idx / kDMaxChunks) % kDW, c = idx % kDMaxChunks;
+                float v = 0.f;
+                if (idx < E) {
+                    // chunks a warp never had keep whatever the table held: mask them by count
+                    const int cu0r = (int)((long long)r * NU / P), cu1r = (int)((long long)(r + 1) * NU / P);
+                    const int a0 = cu0r + (int)((long long)w * (cu1r - cu0r) / kDW);
+                    const int a1 = cu0r + (int)((long long)(w + 1) * (cu1r - cu0r) / kDW);
+                    const int nc = min(kDMaxChunks, (a1 - a0 + kDChunkUnits - 1) / kDChunkUnits);
+                    if (c < nc) v = ex2(sh.cm[r][w][c] - Mr) * sh.cs[r][w][c];
+                }
+                float incl = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const float t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const unsigned mh = __ballot_sync(0xFFFFFFFFu, v > 0.f && run + incl > target);
+                const unsigned ml = __ballot_sync(0xFFFFFFFFu, v > 0.f);
+                if (ml) {
+                    const int l = 31 - __clz(ml);
+                    last = e + l;
+                    lbase = run + __shfl_sync(0xFFFFFFFFu, incl - v, l);
+                }
+                if (mh) {
+                    const int l = __ffs(mh) - 1;
+                    hit = e + l;
+                    base = run + __shfl_sync(0xFFFFFFFFu, incl - v, l);
+                }
+                run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            }
+            if (hit < 0) {           // rounding left no crossing: last chunk with mass, last token with mass
+                hit = last;
+                base = lbase;
+                target = INFINITY;
+            }
+            if (hit >= 0) {
+                const int r = hit / (kDW * kDMaxChunks), w = (hit / kDMaxChunks) % kDW, c = hit % kDMaxChunks;
+                const int cu0r = (int)((long long)r * NU / P), cu1r = (int)((long long)(r + 1) * NU / P);
+                const int a0 = cu0r + (int)((long long)w * (cu1r - cu0r) / kDW);
+                const int a1 = cu0r + (int)((long long)(w + 1) * (cu1r - cu0r) / kDW);
+                const int u0 = a0 + c * kDChunkUnits, u1 = min(a1, u0 + kDChunkUnits);
+                const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(p.z) + (long long)b * p.row_stride;
+                tok = warp_scan_select<8>(u0, u1, p.V, base, target, [&](int u, float(&wt)[8]) {
+                    const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + u);
+                    const uint32_t qw[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 z = unpack2(bclamp2(qw[j]));
+                        wt[2 * j] = ex2(fmaf(z.x, kLog2e, -Mr));
+                        wt[2 * j + 1] = ex2(fmaf(z.y, kLog2e, -Mr));
+                    }
+                });
+            }
+        }
+        if (lane == 0) {
+            if (rowbad) atomicOr(p.st.status, ADASD_STATUS_NAN);
+            p.H_out[b] = H;
+            if (p.lse_out) p.lse_out[b] = lse;
+            if (sampling) p.token_out[b] = tok;
+            const bool stop = H > p.st.T_G[b];   // strict; NaN never stops
+            if (p.stop_out) p.stop_out[b] = stop ? 1 : 0;
+            if (p.draft_len) p.draft_len[b] += 1;
+            if (p.active && stop) p.active[b] = 0;
+        }
+    }
+}
+
+}  // namespace adasd
