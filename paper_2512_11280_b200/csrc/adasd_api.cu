@@ -23,8 +23,8 @@ struct adasd_ctx {
     Scratch sc;
     std::vector<void*> allocs;
     int sm_count;
-    // cluster kernels, one configuration per mode (AdaSD: warp-specialised kernel, vanilla:
-    // streaming cluster kernel); iter == 0 means not usable for this V / dtype
+    // warp-specialised verification kernel, one configuration per mode (AdaSD, vanilla);
+    // iter == 0 means not usable for this V / dtype
     struct Fast {
         int iter;             // iterations per warp and row (template parameter)
         int cs;               // CTAs per cluster
@@ -92,7 +92,7 @@ int launch_cluster(void (*kernel)(P), const P& params, long long clusters, int c
     return ADASD_OK;
 }
 
-// ---- streaming cluster kernel: configuration and launch ---------------------------------
+// ---- warp-specialised verification kernel: configuration and launch ----------------------
 template <typename K>
 int kernel_occupancy(K kern, int threads, int cs, int smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -129,16 +129,14 @@ int kernel_static_smem(K kern) {
     return (int)fa.sharedSizeBytes;
 }
 
-// AdaSD mode runs the warp-specialised kernel, vanilla mode the streaming cluster kernel.
+// Both modes run the warp-specialised kernel.
 template <int ITER, int MODE>
 int fast_occupancy(int cs, int smem) {
-    if (MODE == MODE_ADASD) return kernel_occupancy(spec_verify_kernel<ITER>, kSThreads, cs, smem);
-    return kernel_occupancy(cluster_verify_kernel<ITER, MODE_VANILLA>, kCThreads, cs, smem);
+    return kernel_occupancy(spec_verify_kernel<ITER, MODE>, kSThreads, cs, smem);
 }
 template <int ITER, int MODE>
 int fast_static_smem() {
-    if (MODE == MODE_ADASD) return kernel_static_smem(spec_verify_kernel<ITER>);
-    return kernel_static_smem(cluster_verify_kernel<ITER, MODE_VANILLA>);
+    return kernel_static_smem(spec_verify_kernel<ITER, MODE>);
 }
 
 #define ADASD_ITER_SWITCH(iter, CALL, fail)  \
@@ -170,44 +168,26 @@ int fast_static_smem_iter(int iter) {
 }
 
 // Chooses, for one mode, the cluster size that covers the most SMs among those whose per-CTA
-// slice fits on chip: the kept 2^t values (registers first, shared memory for the rest) plus
-// a ring of at least one position.  bf16 rows of a multiple of 8 elements only.
+// slice fits on chip: two position buffers per compute warp, iter * 512 bytes per row (the
+// 2^t values live in registers or are worked out again).  bf16 rows of a multiple of 8
+// elements only.
 template <int MODE>
 void fast_setup_mode(adasd_ctx* c, size_t smem_optin) {
     adasd_ctx::Fast& f = c->fast[MODE];
     f.iter = 0;
     const int V = c->cfg.V;
     if (c->cfg.dtype != ADASD_BF16 || (V & 7) != 0 || V < 8192) return;
-    const int warps = (MODE == MODE_ADASD) ? kSW : kCW;          // warps that split a CTA's slice
-    const int reg_iter = (MODE == MODE_ADASD) ? kSRegIter : kCRegIter;
     const int NU = V >> 3;
     int best_score = 0;
     for (int cs = kCMaxCluster; cs >= 1; --cs) {
         if (c->cfg.cluster_size != 0 && c->cfg.cluster_size != cs) continue;
         const int ncu = (NU + cs - 1) / cs, nwi = (ncu + 31) / 32;
-        const int I_lo = nwi / warps, rem = nwi % warps, iter = I_lo + (rem ? 1 : 0);
-        if (iter < 1 || iter > kCMaxIter) continue;
+        const int I_lo = nwi / kSW, rem = nwi % kSW, iter = I_lo + (rem ? 1 : 0);
+        if (iter < 1 || iter > kSMaxIter) continue;
         const int st = fast_static_smem_iter<MODE>(iter);
         if (st < 0) continue;
-        int NS, smem, stash_off;
-        if (MODE == MODE_ADASD) {
-            // two position buffers per compute warp, iter * 512 bytes per row; nothing else
-            NS = 2;
-            smem = warps * iter * 2048;
-            stash_off = 0;
-            if (smem > (int)smem_optin - st - 1024) continue;
-        } else {
-            const int KR = std::min(iter, reg_iter);
-            int stash_slots = 0;
-            if (iter > KR) stash_slots = (iter - 1 - KR) * warps + ((iter - 1 < I_lo) ? warps : rem);
-            const int stash_bytes = stash_slots * kCSlotBytes;
-            const int avail = (int)smem_optin - st - stash_bytes - 1024;
-            const int n_stg = (iter + 1) / 2;
-            NS = std::min({kCMaxSlots, avail / (warps * kCSlotBytes), 2 * n_stg});
-            if (NS < n_stg) continue;
-            smem = NS * warps * kCSlotBytes + stash_bytes;
-            stash_off = NS * warps * kCSlotBytes;
-        }
+        const int smem = kSW * iter * 2048;
+        if (smem > (int)smem_optin - st - 1024) continue;
         const int ncl = fast_occupancy_iter<MODE>(iter, cs, smem);
         const int score = ncl * cs;
         if (score > best_score) {
@@ -215,8 +195,6 @@ void fast_setup_mode(adasd_ctx* c, size_t smem_optin) {
             f.iter = iter;
             f.cs = cs;
             f.smem = smem;
-            f.geom.NS = NS;
-            f.geom.stash_off = stash_off;
             f.geom.ncl = ncl;
         }
     }
@@ -260,7 +238,7 @@ int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
     cudaLaunchConfig_t lc;
     memset(&lc, 0, sizeof(lc));
     lc.gridDim = dim3((unsigned)(gq.ncl * f.cs), 1, 1);
-    lc.blockDim = dim3((unsigned)(MODE == MODE_ADASD ? kSThreads : kCThreads), 1, 1);
+    lc.blockDim = dim3((unsigned)kSThreads, 1, 1);
     lc.dynamicSmemBytes = (size_t)f.smem;
     lc.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -270,11 +248,7 @@ int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    if (MODE == MODE_ADASD) {
-        CUDA_TRY(cudaLaunchKernelEx(&lc, spec_verify_kernel<ITER>, p, gq));
-    } else {
-        CUDA_TRY(cudaLaunchKernelEx(&lc, cluster_verify_kernel<ITER, MODE_VANILLA>, p, gq));
-    }
+    CUDA_TRY(cudaLaunchKernelEx(&lc, spec_verify_kernel<ITER, MODE>, p, gq));
     return ADASD_OK;
 }
 

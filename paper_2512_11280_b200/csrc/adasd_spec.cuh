@@ -1,22 +1,30 @@
-// Warp-specialised AdaSD verification kernel for sm_100a.
+// Warp-specialised verification kernel for sm_100a (AdaSD mode and vanilla speculative
+// sampling mode).
 //
-// Same data path as the streaming cluster kernel (persistent clusters, per-warp slot rings
-// filled by 1-D bulk copies, 2^t values kept in registers and shared memory, every logit row
-// read from HBM once), but the irregular work is taken off the arithmetic warps:
+// Persistent thread-block clusters; a position (b,i) = target row p_i + draft row q_i (bf16).
+// The CTAs of a cluster split both rows into contiguous slices, the compute warps of a CTA
+// split the CTA's slice into contiguous runs of "iterations" (one iteration = 32 lanes x 16
+// bytes of each row).  Every logit row is read from HBM exactly once, by 1-D bulk copies
+// (cp.async.bulk) into per-warp buffers that hold two whole positions; the copy of position
+// n + 2 is issued the moment position n is done with, so HBM never waits for the arithmetic.
+// Values live in the log2 domain: t = z log2 e - M, 2^t kept in registers for the first
+// iterations and worked out again from the buffer for the rest.
 //
-//  * 10 COMPUTE warps per CTA do nothing but the three passes over their share of a position
-//    (maxima; 2^t, S and T; (p+q) log2 (p+q)), the refill of their own ring slots and, for
-//    the one warp that holds it, the inverse-CDF crossing.
+//  * 10 COMPUTE warps per CTA do nothing but the passes over their share of a position
+//    (A: maxima and flags; B: 2^t, S = sum 2^t and T = sum 2^t t; C: (p+q) log2 (p+q) in
+//    AdaSD mode, the residual mass max(0, p - q) of a rejected row in vanilla mode), the
+//    refill of their own buffers and, for the one warp that holds it, the inverse-CDF crossing.
 //  * 1 CONTROL warp per CTA finds the cluster's positions, folds the warp partials into the
 //    CTA's totals, exchanges them with the other CTAs of the cluster (st.async into their
 //    shared memory, counted on their mbarriers: no cluster-wide barrier in the loop) and
-//    turns the row totals into two small messages per compute warp: its scale factors, then
-//    whether it holds the inverse-CDF crossing.
+//    turns the row totals into two small messages per compute warp: its scale factors (and,
+//    vanilla, whether the row was accepted), then whether it holds the inverse-CDF crossing.
 //  * 1 TAIL warp (leader CTA) finalises each position once the compute warps' sums are in,
 //    draws the sequence's ticket and runs the tails (KDE/Bayes, accept scan, list appends,
-//    T_G) of completed sequences, off everybody's critical path.
+//    T_G; vanilla: longest accepted prefix) of completed sequences, off everybody's critical
+//    path; AdaSD tails are handed to the idle tail warps of the cluster's other CTAs.
 //
-// Every wait (slot filled, partials in, totals in, message ready, sums in, queue) is bounded:
+// Every wait (buffer filled, partials in, totals in, message ready, sums in, queue) is bounded:
 // a warp whose wait expires sets ADASD_STATUS_TIMEOUT, stops waiting and copying, and walks
 // through the rest of the protocol, so the kernel always ends.
 #pragma once
@@ -30,6 +38,7 @@ constexpr int kSCtl = kSW;                       // warp index of the control wa
 constexpr int kSTail = kSW + 1;                  // warp index of the tail warp
 constexpr int kSThreads = (kSW + 2) * 32;        // 384: leaves 168 registers per thread
 constexpr int kSRegIter = 6;                     // iterations whose 2^t values stay in registers
+constexpr int kSMaxIter = 10;                    // largest number of iterations per warp and row
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
 constexpr int kSPosRing = 16;                    // positions the control warp keeps described
 constexpr int kSWorkQ = 16;                      // tail work queue entries per CTA
@@ -49,7 +58,8 @@ struct __align__(16) PosCtx {
 // What a compute warp needs after the exchange: p = 2^t_p * at, q = 2^t_q * ad; and, if it
 // holds the inverse-CDF crossing (sel), the weight before its share and the target.
 struct __align__(16) WarpMsg {
-    float at, ad, ft, pad0;       // first part: ready when scal_bar completes
+    float at, ad, ft;             // first part: ready when scal_bar completes
+    int32_t act;                  // vanilla: 0 nothing left to do, 1 sample from p, 2 residual pass
     float target;                 // second part: ready when sel_bar completes
     int32_t sel;
     float base;
@@ -62,12 +72,16 @@ struct __align__(16) SpecShared {
     RowPart ctab[2][kCMaxCluster];    // every CTA's totals (written over DSMEM), by parity
     WarpMsg wmsg[2][kCW];
     float4 tabC[kSFinRing][kCTab];    // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q, token or -1), by position
-    float fin[kSFinRing][8];          // leader: row totals kept for finalisation
+    float fin[kSFinRing][12];         // leader: row totals (and alpha, accept flag) kept for finalisation
+    float rw[kCW];                    // vanilla: residual mass of each compute warp's share
+    float4 rtab[kCMaxCluster];        // vanilla: every CTA's residual mass (written over DSMEM)
     unsigned long long entry_bar[2];  // one arrival per compute warp: wtab[par] complete
     unsigned long long ctab_bar[2];   // CS * 32 bytes from the control warps of the cluster: ctab[par] complete
     unsigned long long scal_bar[2];   // 1 arrival: first part of wmsg[par] ready
     unsigned long long sel_bar[2];    // 1 arrival: second part of wmsg[par] ready
     unsigned long long c_bar[kSFinRing];   // leader: 16 bytes from every compute warp of the cluster: tabC complete
+    unsigned long long resid_bar;     // vanilla: one arrival per compute warp: rw complete
+    unsigned long long r_bar;         // vanilla: CS * 16 bytes from the control warps of the cluster: rtab complete
     unsigned long long bar[kCW][2];   // per compute warp: "position buffer filled" barriers
     int32_t n_issued;                 // leader: positions whose messages have been sent
     int32_t n_final;                  // leader: number of positions of this cluster, -1 until known
@@ -228,7 +242,7 @@ __device__ __forceinline__ void verify_tail_warp(const TailConfig& cfg, const Ta
 }
 
 // ------------------------------------------------------------------------------------
-template <int ITER>
+template <int ITER, int MODE>
 __global__ void __launch_bounds__(kSThreads, 1)
 spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
     constexpr int KR = ITER < kSRegIter ? ITER : kSRegIter;   // iterations kept in registers
@@ -266,6 +280,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             mbar_init(reinterpret_cast<uint64_t*>(&sh.sel_bar[k]), 1);
         }
         for (int k = 0; k < kSFinRing; ++k) mbar_init(reinterpret_cast<uint64_t*>(&sh.c_bar[k]), 1);
+        mbar_init(reinterpret_cast<uint64_t*>(&sh.resid_bar), kSW);
+        mbar_init(reinterpret_cast<uint64_t*>(&sh.r_bar), 1);
     }
     if (warp < kSW && lane == 0)
         for (int s = 0; s < 2; ++s) mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][s]), 1);
@@ -540,16 +556,16 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         };
 
         // Run by the warp that holds the crossing: first element (index order: iteration, lane,
-        // element) of the target row where base + f * running weight exceeds target, else the
-        // last element with weight.
-        auto select_kept = [&](int n, float base, float f, float target) -> int {
+        // element) where base + f * running weight exceeds target, else the last element with
+        // weight.  vals(k, v) fills the 8 weights of this lane's unit of iteration k.
+        auto select_kept = [&](float base, float f, float target, auto vals) -> int {
             float ls[ITER], tot[ITER];
 #pragma unroll
             for (int k = 0; k < ITER; ++k) {
                 ls[k] = 0.f;
                 if (k_on(k)) {
-                    float v[8], d[8];
-                    load_kept(k, n, false, v, d);
+                    float v[8];
+                    vals(k, v);
                     ls[k] = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
                 }
             }
@@ -581,8 +597,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
 #pragma unroll
             for (int k = 0; k < ITER; ++k) {
                 if (k == ksel) {          // same for the whole warp
-                    float d[8];
-                    load_kept(k, n, false, v, d);
+                    vals(k, v);
                     lsum = ls[k];
                 }
             }
@@ -636,38 +651,80 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             wait_cta(&sh.scal_bar[par], ph);
             const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft
 
-            // pass C: sum (p+q) log2 (p+q) and the overlap indicator sum 2^t_p 2^t_q
+            // the target row's 2^t values of iteration k (what y_i ~ p_i is drawn from)
+            auto vals_p = [&](int k, float(&v)[8]) {
+                float d[8];
+                load_kept(k, n, false, v, d);
+            };
             float A = 0.f, PQ = 0.f;
-            if (!bonus) {
-                float2 A2 = make_float2(0.f, 0.f), PQ2 = make_float2(0.f, 0.f);
-                const float2 at2 = make_float2(m0.x, m0.x), ad2 = make_float2(m0.y, m0.y);
-                const float2 tiny2 = make_float2(kTiny, kTiny);
+            int tok = -1;
+            if (MODE == MODE_ADASD) {
+                // pass C: sum (p+q) log2 (p+q) and the overlap indicator sum 2^t_p 2^t_q
+                if (!bonus) {
+                    float2 A2 = make_float2(0.f, 0.f), PQ2 = make_float2(0.f, 0.f);
+                    const float2 at2 = make_float2(m0.x, m0.x), ad2 = make_float2(m0.y, m0.y);
+                    const float2 tiny2 = make_float2(kTiny, kTiny);
 #pragma unroll
-                for (int k = 0; k < ITER; ++k) {
-                    if (k_on(k)) {
-                        float a[8], d[8];
-                        load_kept(k, n, true, a, d);
+                    for (int k = 0; k < ITER; ++k) {
+                        if (k_on(k)) {
+                            float a[8], d[8];
+                            load_kept(k, n, true, a, d);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float2 a2 = make_float2(a[2 * j], a[2 * j + 1]);
-                            const float2 d2 = make_float2(d[2 * j], d[2 * j + 1]);
-                            const float2 pp = __ffma2_rn(a2, at2, tiny2);
-                            const float2 ss = __ffma2_rn(d2, ad2, pp);
-                            const float2 ll = make_float2(lg2(ss.x), lg2(ss.y));
-                            A2 = __ffma2_rn(ss, ll, A2);
-                            PQ2 = __ffma2_rn(a2, d2, PQ2);
+                            for (int j = 0; j < 4; ++j) {
+                                const float2 a2 = make_float2(a[2 * j], a[2 * j + 1]);
+                                const float2 d2 = make_float2(d[2 * j], d[2 * j + 1]);
+                                const float2 pp = __ffma2_rn(a2, at2, tiny2);
+                                const float2 ss = __ffma2_rn(d2, ad2, pp);
+                                const float2 ll = make_float2(lg2(ss.x), lg2(ss.y));
+                                A2 = __ffma2_rn(ss, ll, A2);
+                                PQ2 = __ffma2_rn(a2, d2, PQ2);
+                            }
                         }
                     }
+                    A = warp_sum(A2.x + A2.y);
+                    PQ = warp_sum(PQ2.x + PQ2.y);
                 }
-                A = warp_sum(A2.x + A2.y);
-                PQ = warp_sum(PQ2.x + PQ2.y);
+                // y_i ~ p_i: the control warp says (a little later than the scale factors) whether
+                // this warp holds the crossing
+                wait_cta(&sh.sel_bar[par], ph);
+                const float4 m1 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp].target);   // target, sel, base
+                if (__float_as_int(m1.y) != 0) tok = select_kept(m1.z, m0.z, m1.x, vals_p);
+            } else {
+                // vanilla: an accepted row needs nothing more; the bonus row draws from p; a rejected
+                // row draws from the residual max(0, p - q) / R, whose mass this warp now adds up
+                const int act = __float_as_int(m0.w);
+                const float at = m0.x, ad = m0.y;
+                auto vals_r = [&](int k, float(&v)[8]) {
+                    float a[8], d[8];
+                    load_kept(k, n, true, a, d);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = fmaxf(fmaf(a[j], at, -d[j] * ad), 0.f);
+                };
+                if (act == 2) {
+                    float r = 0.f;
+#pragma unroll
+                    for (int k = 0; k < ITER; ++k) {
+                        if (k_on(k)) {
+                            float v[8];
+                            vals_r(k, v);
+                            r += ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+                        }
+                    }
+                    r = warp_sum(r);
+                    if (lane == 0) {
+                        sh.rw[warp] = r;
+                        mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.resid_bar));
+                    }
+                    __syncwarp();
+                }
+                if (act != 0) {
+                    wait_cta(&sh.sel_bar[par], ph);
+                    const float4 m1 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp].target);   // target, sel, base
+                    const int sel = __float_as_int(m1.y);
+                    if (sel == 1) tok = select_kept(m1.z, m0.z, m1.x, vals_p);
+                    else if (sel == 2) tok = select_kept(m1.z, 1.f, m1.x, vals_r);
+                }
             }
-            // y_i ~ p_i: the control warp says (a little later than the scale factors) whether this
-            // warp holds the crossing
-            wait_cta(&sh.sel_bar[par], ph);
-            const float4 m1 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp].target); // target, sel, base
-            int tok = -1;
-            if (__float_as_int(m1.y) != 0) tok = select_kept(n, m1.z, m0.z, m1.x);
             // the buffer of position n is free: fetch position n + 2 into it
             __syncwarp();
             issue_pos(n + 2);
@@ -697,6 +754,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             return __shfl_sync(0xFFFFFFFFu, v, 0);
         };
         int n = 0;
+        uint32_t nres = 0;                        // residual exchanges so far (phase of their barriers)
         while (sh.pc[n & (kSPosRing - 1)].pos < total) {
             const int par = n & 1;
             const uint32_t ph = (uint32_t)(n >> 1) & 1u;
@@ -709,7 +767,27 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 set_pos(n + 3, r);
                 lastp = r;
             }
-            const float u_samp = __ldg(p.u_target + sh.pc[n & (kSPosRing - 1)].pos);
+            // per-position scalars, fetched before the wait so that they are there after it
+            const PosCtx& pcn = sh.pc[n & (kSPosRing - 1)];
+            const bool bonus = pcn.bonus != 0;
+            float u_samp, u_acc = 0.f, ztx = 0.f, zdx = 0.f;
+            bool x_ok = false;
+            if (MODE == MODE_ADASD) {
+                u_samp = __ldg(p.u_target + pcn.pos);
+            } else {
+                const int b = pcn.pos / K1, i = pcn.pos - b * K1;
+                u_samp = __ldg(p.u_resample + b);
+                if (!bonus) {
+                    const size_t idd = (size_t)b * Kmax + i;
+                    u_acc = __ldg(p.u_accept + idd);
+                    const int xi = __ldg(p.x + idd);
+                    x_ok = xi >= 0 && xi < p.V;
+                    if (x_ok) {
+                        ztx = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.zt)[(long long)b * p.t_seq + (long long)i * p.t_row + xi]);
+                        zdx = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.zd)[(long long)b * p.d_seq + (long long)i * p.d_row + xi]);
+                    }
+                }
+            }
 
             // the CTA's totals from its compute warps, sent to every CTA of the cluster
             wait_cta(&sh.entry_bar[par], ph);
@@ -761,29 +839,48 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const float st_c = cft * e0.y;                    // CTA sums of the target row, scaled to Mt
             const float St = sum8(st_c), Sd = sum8(cfd * e1.x);
 
+            // vanilla: alpha = min(1, p(x) / q(x)) at the draft token, and what is left to do
+            const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(e1.z));
+            const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL);
+            float alpha = 0.f;
+            bool van_accept = true;
+            int act = 1;                          // AdaSD: every row draws y_i ~ p_i
+            if (MODE == MODE_VANILLA) {
+                if (!bonus) {
+                    if (x_ok) {
+                        const float a = fmaf(fmaxf(ztx, ADASD_FLOOR_BF), kLog2e, -Mt) - lg2(St);
+                        const float q = fmaf(fmaxf(zdx, ADASD_FLOOR_BF), kLog2e, -Md) - lg2(Sd);
+                        alpha = fminf(1.f, ex2(a - q));
+                        if (!(ex2(q) > 0.f)) alpha = 1.f;   // q(x) = 0 cannot have been drafted
+                    }
+                    van_accept = u_acc < alpha;
+                }
+                act = bad ? 0 : (bonus ? 1 : (van_accept ? 0 : 2));
+            }
+
             // first message per compute warp (lane w): its scale factors; pass C starts on it
             const float ftw = ex2(w0.x - Mt), fdw = ex2(w0.w - Md);
             const float at = __fdividef(ftw, St), ad = __fdividef(fdw, Sd);
-            if (lane < kSW) *reinterpret_cast<float4*>(&sh.wmsg[par][lane]) = make_float4(at, ad, ftw, 0.f);
+            if (lane < kSW) *reinterpret_cast<float4*>(&sh.wmsg[par][lane]) = make_float4(at, ad, ftw, __int_as_float(act));
             __syncwarp();
             if (lane == 0) mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.scal_bar[par]));
 
-            // off the critical path: T totals and flags for the finaliser, then the second message:
-            // which warp holds the crossing of target = u * S_t in index order (CTA by CTA, then
-            // warp by warp)
+            // Off the critical path: T totals for the finaliser, then the second message.
             const float Tt = sum8(cft * fmaf(cdt, e0.y, e0.z)), Td = sum8(cfd * fmaf(cdd, e1.x, e1.y));
-            const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(e1.z));
-            const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL);
+            // Which warp holds the crossing of `target`
+            // in index order (CTA by CTA, then warp by warp), given the weight cw of CTA `lane` and
+            // the weight ww of this CTA's compute warp `lane`; `kind` says what the warp scans.
             int sel = 0;
-            float base = 0.f, target = u_samp * St;
-            if (!bad) {
-                float incl = st_c;
+            float base = 0.f, target = 0.f;
+            auto locate = [&](float cw, float ww, float tgt, int kind) {
+                target = tgt;
+                float incl = cw;
 #pragma unroll
                 for (int o = 1; o < 8; o <<= 1) {
                     const float t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
                     if (lane >= o) incl += t;
                 }
-                const bool mass = lane < CS && st_c > 0.f;
+                const bool mass = lane < CS && cw > 0.f;
                 int cstar = -1;
                 const unsigned mc = __ballot_sync(0xFFFFFFFFu, mass && incl > target);
                 if (mc) {
@@ -793,9 +890,9 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     if (ml) cstar = 31 - __clz(ml);
                     target = INFINITY;
                 }
-                const float cbase = __shfl_sync(0xFFFFFFFFu, incl - st_c, max(cstar, 0));
+                const float cbase = __shfl_sync(0xFFFFFFFFu, incl - cw, max(cstar, 0));
                 if (cstar == rank) {
-                    const float w = (lane < kSW) ? ftw * w0.y : 0.f;
+                    const float w = (lane < kSW) ? ww : 0.f;
                     float winc = w;
 #pragma unroll
                     for (int o = 1; o < 16; o <<= 1) {
@@ -812,11 +909,31 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                         target = INFINITY;
                     }
                     if (lane == wsel) {
-                        sel = 1;
+                        sel = kind;
                         base = cbase + (winc - w);
                     }
                 }
+            };
+            bool from_p = (act == 1);
+            if (MODE == MODE_VANILLA && act == 2) {
+                // residual mass: warp sums -> CTA sum -> every CTA of the cluster
+                const uint32_t rph = nres & 1u;
+                ++nres;
+                wait_cta(&sh.resid_bar, rph);
+                const float rwv = (lane < kSW) ? sh.rw[lane] : 0.f;
+                const float r_cta = warp_sum(rwv);
+                if (lane == 0) mbar_expect_tx(reinterpret_cast<uint64_t*>(&sh.r_bar), (uint32_t)(CS * 16));
+                __syncwarp();
+                if (lane < CS)
+                    st_async_v4(mapa_u32(&sh.rtab[rank], (uint32_t)lane), make_float4(r_cta, 0.f, 0.f, 0.f),
+                                mapa_u32(&sh.r_bar, (uint32_t)lane));
+                wait_cta(&sh.r_bar, rph);
+                const float rc = (lane < CS) ? sh.rtab[lane].x : 0.f;
+                const float R = sum8(rc);
+                if (R > 0.f && alive) locate(rc, rwv, u_samp * R, 2);
+                else from_p = true;               // no residual mass: draw from p
             }
+            if (from_p && !bad) locate(st_c, ftw * w0.y, u_samp * St, 1);
             if (lane < kSW)
                 *reinterpret_cast<float4*>(&sh.wmsg[par][lane].target) = make_float4(target, __int_as_float(sel), base, 0.f);
             if (leader && lane == 0) {
@@ -828,11 +945,16 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 f[4] = Sd;
                 f[5] = Td;
                 f[6] = __uint_as_float(fl | (alive ? 0u : 1u));
+                f[7] = alpha;
+                f[8] = van_accept ? 1.f : 0.f;
             }
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.sel_bar[par]));
-                if (leader) *reinterpret_cast<volatile int32_t*>(&sh.n_issued) = n + 1;
+                if (leader) {
+                    __threadfence_block();
+                    *reinterpret_cast<volatile int32_t*>(&sh.n_issued) = n + 1;
+                }
             }
             ++n;
         }
@@ -885,6 +1007,13 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                         atomicOr(p.st.status, ADASD_STATUS_NAN);
                         tok = -1;
                     }
+                    if (MODE == MODE_VANILLA) {
+                        if (!bonus) {
+                            p.sc.van_flag[idd] = (sh.fin[par][8] != 0.f && !bad) ? 1 : 0;
+                            if (p.alpha_out) p.alpha_out[idd] = bad ? NAN : sh.fin[par][7];
+                        }
+                        p.sc.van_tok[idt] = tok;
+                    } else {
                     const float lSt = lg2(St), lSd = lg2(Sd);
                     const float Hbt = lSt - Tt / St, Hbd = lSd - Td / Sd;      // entropies in bits
                     float Ht = kLn2 * Hbt, lse_t = kLn2 * (Mt + lSt);
@@ -911,6 +1040,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                         if (p.user.lse_d) p.user.lse_d[idd] = lse_d;
                         if (p.user.jsd) p.user.jsd[idd] = jsd;
                         if (p.user.dist) p.user.dist[idd] = dist;
+                    }
                     }
                     __threadfence();
                     const unsigned ticket = atomicAdd(p.sc.ticket + b, 1u);
@@ -971,7 +1101,19 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 if (go <= 0) break;
                 const int done_b = finalize(m);
                 if (done_b >= 0) {
-                    if (CS > 1) {
+                    if (MODE == MODE_VANILLA) {
+                        // longest accepted prefix, then the token drawn at the first rejection
+                        // (or the bonus token)
+                        __threadfence();
+                        const int kt = window(done_b);
+                        const bool rej = lane < kt && __ldcg(p.sc.van_flag + (size_t)done_b * Kmax + lane) == 0;
+                        const unsigned mr = __ballot_sync(0xFFFFFFFFu, rej);
+                        if (lane == 0) {
+                            const int w = mr ? (__ffs(mr) - 1) : kt;
+                            p.accept_len[done_b] = w;
+                            p.next_token[done_b] = __ldcg(p.sc.van_tok + (size_t)done_b * K1 + w);
+                        }
+                    } else if (CS > 1) {
                         dispatch(done_b);
                     } else {
                         __threadfence();

@@ -88,6 +88,16 @@ def test_small_and_ragged_vocabularies(torch, V, dtype, cs):
     run_lockstep(wl, cluster_size=cs, min_kde_samples=3)
 
 
+@pytest.mark.parametrize("cs", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_streaming_kernels_at_every_cluster_size(torch, cs):
+    # bf16 rows of a multiple of 8 logits take the warp-specialised kernels: 20008 logits give
+    # every cluster size a different split (10 iterations per warp down to 1, ragged last unit),
+    # in AdaSD mode and in vanilla mode (C3 runs both)
+    wl = synth.WORKLOADS["C3"].scaled(name=f"stream_cs{cs}", B=5, K=3, V=20008, rounds=8)
+    rep = run_lockstep(wl, cluster_size=cs, min_kde_samples=3)
+    assert len(rep.vanilla_accept_hist) >= 2
+
+
 def test_c2_single_stream_adaptive_window(torch):
     wl = synth.WORKLOADS["C2"].scaled(rounds=40)
     rep = run_lockstep(wl)
