@@ -8,7 +8,7 @@
 // (cp.async.bulk) into per-warp buffers that hold two whole positions; the copy of position
 // n + 2 is issued the moment position n is done with, so HBM never waits for the arithmetic.
 // Values live in the log2 domain: t = z log2 e - M, 2^t kept in registers for the first
-// iterations and worked out again from the buffer for the rest.
+// iterations and, for the rest, parked in the buffer over logits that have been used up.
 //
 //  * 10 COMPUTE warps per CTA do nothing but the passes over their share of a position
 //    (A: maxima and flags; B: 2^t, S = sum 2^t and T = sum 2^t t; C: (p+q) log2 (p+q) in
@@ -39,6 +39,9 @@ constexpr int kSTail = kSW + 1;                  // warp index of the tail warp
 constexpr int kSThreads = (kSW + 2) * 32;        // 384: leaves 168 registers per thread
 constexpr int kSRegIter = 6;                     // iterations whose 2^t values stay in registers
 constexpr int kSMaxIter = 10;                    // largest number of iterations per warp and row
+// Iteration k >= kSRegIter parks its 2^t values in the buffer pieces of iterations 2 (k - kSRegIter)
+// and 2 (k - kSRegIter) + 1, which must have been consumed before it: 2 (k - kSRegIter) + 1 < k.
+static_assert(2 * (kSMaxIter - 1 - kSRegIter) + 1 < kSMaxIter - 1, "parked 2^t values would overwrite unread logits");
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
 constexpr int kSPosRing = 16;                    // positions the control warp keeps described
 constexpr int kSWorkQ = 16;                      // tail work queue entries per CTA
@@ -515,6 +518,17 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                             et[k < KR ? k : 0][j] = e1[j];
                             ed[k < KR ? k : 0][j] = e2[j];
                         }
+                    } else {
+                        // no register left: the values go over logits this lane has already turned
+                        // into 2^t values (two 512-byte pieces of each row per iteration)
+                        float4* st = reinterpret_cast<float4*>(const_cast<unsigned char*>(sb) + (k - KR) * 1024);
+                        st[0] = make_float4(e1[0], e1[1], e1[2], e1[3]);
+                        st[32] = make_float4(e1[4], e1[5], e1[6], e1[7]);
+                        if (!BONUS) {
+                            float4* sd = reinterpret_cast<float4*>(const_cast<unsigned char*>(sb) + kRowB + (k - KR) * 1024);
+                            sd[0] = make_float4(e2[0], e2[1], e2[2], e2[3]);
+                            sd[32] = make_float4(e2[4], e2[5], e2[6], e2[7]);
+                        }
                     }
                 }
             }
@@ -528,9 +542,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 sB[3] = warp_sum(Td.x + Td.y);
             }
         };
-        // The 2^t values of iteration k (compile-time k after unrolling): kept ones from
-        // registers, the others worked out again from the logits, which stay in the buffer until
-        // pass C is over (ex2 is cheap; shared-memory bandwidth for a second copy is not).
+        // The 2^t values of iteration k (compile-time k after unrolling): from registers, or from
+        // where pass B left them in the position's buffer.
         auto load_kept = [&](int k, int n, bool with_d, float (&a)[8], float (&b)[8]) {
             if (k < KR) {
 #pragma unroll
@@ -540,14 +553,13 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 }
             } else {
                 const unsigned char* sb = buf_of(n);
-                float2 s0 = make_float2(0.f, 0.f), s1 = s0;
-                uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
-                mask_unit(k, T);
-                exps(T, make_float2(nmt_w, nmt_w), a, s0, s1);
+                const float4* st = reinterpret_cast<const float4*>(sb + (k - KR) * 1024);
+                const float4 a0 = st[0], a1 = st[32];
+                a[0] = a0.x, a[1] = a0.y, a[2] = a0.z, a[3] = a0.w, a[4] = a1.x, a[5] = a1.y, a[6] = a1.z, a[7] = a1.w;
                 if (with_d) {
-                    uint4 D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
-                    mask_unit(k, D);
-                    exps(D, make_float2(nmd_w, nmd_w), b, s0, s1);
+                    const float4* sd = reinterpret_cast<const float4*>(sb + kRowB + (k - KR) * 1024);
+                    const float4 b0 = sd[0], b1 = sd[32];
+                    b[0] = b0.x, b[1] = b0.y, b[2] = b0.z, b[3] = b0.w, b[4] = b1.x, b[5] = b1.y, b[6] = b1.z, b[7] = b1.w;
                 } else {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) b[j] = 0.f;
@@ -725,7 +737,9 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     else if (sel == 2) tok = select_kept(m1.z, 1.f, m1.x, vals_r);
                 }
             }
-            // the buffer of position n is free: fetch position n + 2 into it
+            // the buffer of position n is free: fetch position n + 2 into it (the bulk copy belongs
+            // to the async proxy and must come after this warp's own stores to the buffer)
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             issue_pos(n + 2);
             // this warp's sums (and the token, if it drew it) go to the leader CTA in one message
