@@ -76,6 +76,12 @@ __global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams 
     if (active) {
         issue(0);
         issue(1);
+        // table entries of chunks this warp does not have: no weight
+        if (lane >= nch && lane < kDMaxChunks) {
+            DraftShared* r0 = cluster.map_shared_rank(&sh, 0);
+            r0->cm[rank][warp][lane] = kFloorL;
+            r0->cs[rank][warp][lane] = 0.f;
+        }
         for (int c = 0; c < nch; ++c) {
             bool ok = alive && mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u);
             ok = __all_sync(0xFFFFFFFFu, ok);
@@ -160,68 +166,115 @@ __global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams 
         float H = kLn2 * (lS - T / S), lse = kLn2 * (Mr + lS);
         if (rowbad) H = lse = NAN;
 
-        // x ~ q: which chunk holds the crossing of u * S, in index order (rank, warp, chunk)
+        // x ~ q: the crossing of u * S in index order (rank, warp, chunk): first the warp share
+        // that holds it (entry l of the totals, and l + 32), then the chunk within that share
         int tok = -1;
         const bool sampling = (p.u != nullptr && p.token_out != nullptr);
         if (sampling && !rowbad) {
             float target = __ldg(p.u + b) * S;
-            const int E = NE * kDMaxChunks;
-            float run = 0.f, base = 0.f, lbase = 0.f;
-            int hit = -1, last = -1;
-            for (int e = 0; e < E && hit < 0; e += 32) {
-                const int idx = e + lane;
-                const int r = idx / (kDW * kDMaxChunks), w = (idx / kDMaxChunks) % kDW, c = idx % kDMaxChunks;
-                float v = 0.f;
-                if (idx < E) {
-                    // chunks a warp never had keep whatever the table held: mask them by count
-                    const int cu0r = (int)((long long)r * NU / P), cu1r = (int)((long long)(r + 1) * NU / P);
-                    const int a0 = cu0r + (int)((long long)w * (cu1r - cu0r) / kDW);
-                    const int a1 = cu0r + (int)((long long)(w + 1) * (cu1r - cu0r) / kDW);
-                    const int nc = min(kDMaxChunks, (a1 - a0 + kDChunkUnits - 1) / kDChunkUnits);
-                    if (c < nc) v = ex2(sh.cm[r][w][c] - Mr) * sh.cs[r][w][c];
+            const float w0 = f0 * e0.y, w1 = f1 * e1.y;
+            float i0 = w0, i1 = w1;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float t0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), t1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
+                if (lane >= o) {
+                    i0 += t0;
+                    i1 += t1;
                 }
+            }
+            const float tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31);
+            i1 += tot0;
+            const unsigned h0 = __ballot_sync(0xFFFFFFFFu, w0 > 0.f && i0 > target);
+            const unsigned h1 = __ballot_sync(0xFFFFFFFFu, w1 > 0.f && i1 > target);
+            const unsigned m0 = __ballot_sync(0xFFFFFFFFu, w0 > 0.f), m1 = __ballot_sync(0xFFFFFFFFu, w1 > 0.f);
+            int ent = -1;
+            if (h0) ent = __ffs(h0) - 1;
+            else if (h1) ent = 32 + __ffs(h1) - 1;
+            else {                   // rounding left no crossing: last share with mass, last token with mass
+                if (m1) ent = 32 + 31 - __clz(m1);
+                else if (m0) ent = 31 - __clz(m0);
+                target = INFINITY;
+            }
+            if (ent >= 0) {
+                const float ebase = ent < 32 ? __shfl_sync(0xFFFFFFFFu, i0 - w0, ent)
+                                             : __shfl_sync(0xFFFFFFFFu, i1 - w1, ent - 32);
+                const float* cmf = &sh.cm[0][0][0] + ent * kDMaxChunks;
+                const float* csf = &sh.cs[0][0][0] + ent * kDMaxChunks;
+                const float v = lane < kDMaxChunks ? ex2(cmf[lane] - Mr) * csf[lane] : 0.f;
                 float incl = v;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
+                for (int o = 1; o < 16; o <<= 1) {
                     const float t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
                     if (lane >= o) incl += t;
                 }
-                const unsigned mh = __ballot_sync(0xFFFFFFFFu, v > 0.f && run + incl > target);
-                const unsigned ml = __ballot_sync(0xFFFFFFFFu, v > 0.f);
-                if (ml) {
-                    const int l = 31 - __clz(ml);
-                    last = e + l;
-                    lbase = run + __shfl_sync(0xFFFFFFFFu, incl - v, l);
+                const unsigned ch = __ballot_sync(0xFFFFFFFFu, v > 0.f && ebase + incl > target);
+                const unsigned cl = __ballot_sync(0xFFFFFFFFu, v > 0.f);
+                int c = -1;
+                if (ch) c = __ffs(ch) - 1;
+                else if (cl) {
+                    c = 31 - __clz(cl);
+                    target = INFINITY;
                 }
-                if (mh) {
-                    const int l = __ffs(mh) - 1;
-                    hit = e + l;
-                    base = run + __shfl_sync(0xFFFFFFFFu, incl - v, l);
-                }
-                run += __shfl_sync(0xFFFFFFFFu, incl, 31);
-            }
-            if (hit < 0) {           // rounding left no crossing: last chunk with mass, last token with mass
-                hit = last;
-                base = lbase;
-                target = INFINITY;
-            }
-            if (hit >= 0) {
-                const int r = hit / (kDW * kDMaxChunks), w = (hit / kDMaxChunks) % kDW, c = hit % kDMaxChunks;
-                const int cu0r = (int)((long long)r * NU / P), cu1r = (int)((long long)(r + 1) * NU / P);
-                const int a0 = cu0r + (int)((long long)w * (cu1r - cu0r) / kDW);
-                const int a1 = cu0r + (int)((long long)(w + 1) * (cu1r - cu0r) / kDW);
-                const int u0 = a0 + c * kDChunkUnits, u1 = min(a1, u0 + kDChunkUnits);
-                const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(p.z) + (long long)b * p.row_stride;
-                tok = warp_scan_select<8>(u0, u1, p.V, base, target, [&](int u, float(&wt)[8]) {
-                    const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + u);
-                    const uint32_t qw[4] = {q.x, q.y, q.z, q.w};
+                if (c >= 0) {
+                    const float base = ebase + __shfl_sync(0xFFFFFFFFu, incl - v, c);
+                    const int r = ent / kDW, w = ent % kDW;
+                    const int cu0r = (int)((long long)r * NU / P), cu1r = (int)((long long)(r + 1) * NU / P);
+                    const int a0 = cu0r + (int)((long long)w * (cu1r - cu0r) / kDW);
+                    const int a1 = cu0r + (int)((long long)(w + 1) * (cu1r - cu0r) / kDW);
+                    const int u0 = a0 + c * kDChunkUnits, u1 = min(a1, u0 + kDChunkUnits);
+                    // the chunk again (4 KB, from L2), all of it in flight at once
+                    const uint4* row = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.z) +
+                                                                      (long long)b * p.row_stride);
+                    uint4 Wq[8];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float2 z = unpack2(bclamp2(qw[j]));
-                        wt[2 * j] = ex2(fmaf(z.x, kLog2e, -Mr));
-                        wt[2 * j + 1] = ex2(fmaf(z.y, kLog2e, -Mr));
+                    for (int i = 0; i < 8; ++i) {
+                        const int u = u0 + 32 * i + lane;
+                        Wq[i] = u < u1 ? __ldg(row + u) : make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
                     }
-                });
+                    float run = base;
+                    int last_pos = -1;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (tok < 0 && u0 + 32 * i < u1) {          // same for the whole warp
+                            const int u = u0 + 32 * i + lane;
+                            const uint32_t qw[4] = {Wq[i].x, Wq[i].y, Wq[i].z, Wq[i].w};
+                            float wt[8];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float2 z = unpack2(bclamp2(qw[j]));
+                                wt[2 * j] = ex2(fmaf(z.x, kLog2e, -Mr));
+                                wt[2 * j + 1] = ex2(fmaf(z.y, kLog2e, -Mr));
+                            }
+                            float ls = 0.f;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) ls += wt[j];
+                            float li = ls;
+#pragma unroll
+                            for (int o = 1; o < 32; o <<= 1) {
+                                const float t = __shfl_up_sync(0xFFFFFFFFu, li, o);
+                                if (lane >= o) li += t;
+                            }
+                            float cc = run + (li - ls);
+                            int hit = -1;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                cc += wt[j];
+                                if (wt[j] > 0.f) {
+                                    last_pos = u * 8 + j;
+                                    if (hit < 0 && cc > target) hit = u * 8 + j;
+                                }
+                            }
+                            const unsigned mh = __ballot_sync(0xFFFFFFFFu, hit >= 0);
+                            if (mh) tok = __shfl_sync(0xFFFFFFFFu, hit, __ffs(mh) - 1);
+                            run += __shfl_sync(0xFFFFFFFFu, li, 31);
+                        }
+                    }
+                    if (tok < 0) {
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xFFFFFFFFu, last_pos, o));
+                        tok = last_pos;
+                    }
+                }
             }
         }
         if (lane == 0) {
