@@ -102,6 +102,28 @@ def step_rows(wl) -> dict:
     return {"draft": B * K, "verify": B * (2 * K + 1), "vanilla": B * (2 * K + 1)}
 
 
+# ------------------------------------------------------------------------------ N ranks
+
+def rank_workload(wl, rank: int, sets: int):
+    """The shard of rank `rank`: sequences are independent, so every rank owns its own batch of
+    the workload's shape (weak scaling) from its own seed; no data ever crosses ranks."""
+    return wl.scaled(seed=wl.seed + 1000 * rank, rounds=max(sets, 1))
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum over the ranks of a few timings (the job is as slow as its slowest rank)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_rate(world: int, units_per_rank_step: int, steps: int, ms: float) -> float:
+    """Units all ranks processed in `steps` steps divided by the (max over ranks) time."""
+    return world * units_per_rank_step * steps / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------ our arm
 
 def run_ours(args) -> dict:
@@ -124,7 +146,7 @@ def run_ours(args) -> dict:
     if wl.adaptive_window:
         raise SystemExit("bench.py times the fixed-window workloads (C3, C4)")
     # every rank owns its own sequences: same shapes, different seed
-    wl = wl.scaled(seed=wl.seed + 1000 * rank, rounds=max(args.sets, 1))
+    wl = rank_workload(wl, rank, args.sets)
     B, K, V = wl.B, wl.K, wl.V
     tdt = torch.bfloat16 if wl.dtype == synth.BF16 else torch.float32
     ctx = adasd.Context(B, V, K, dtype=wl.dtype, list_capacity=(args.steps + args.warmup + 64) * K + 64,
@@ -231,10 +253,7 @@ def run_ours(args) -> dict:
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    times = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(times[0]), float(times[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], dist, dev)
 
     rows = step_rows(wl)
     rows_step = sum(rows.values())
@@ -244,7 +263,7 @@ def run_ours(args) -> dict:
     achieved = verify_bytes / (verify_ms * 1e-3) / 1e9
     h2d = (hd.numel() + ht.numel()) * hd.element_size()
     out = {
-        "metric": METRIC, "value": world * rows_step * args.steps / (ms * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": whole_job_rate(world, rows_step, args.steps, ms), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 (bf16 logits, fp32 arithmetic)" if wl.dtype == synth.BF16 else "f32",
@@ -255,7 +274,7 @@ def run_ours(args) -> dict:
                    "sequences_per_gpu": B, "input_sets": nset,
                    "l2": f"inputs larger than L2: {nset} sets of {(2 * K + 1) * B * row_bytes / 1e6:.0f} MB cycled",
                    "hbm_gbs_all_calls": world * rows_step * row_bytes * args.steps / (ms * 1e-3) / 1e9},
-        "e2e": {"value": world * rows_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+        "e2e": {"value": whole_job_rate(world, rows_step, e2e_steps, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": h_out.numel() * 4,
                 "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": args.steps * (K + 2),
