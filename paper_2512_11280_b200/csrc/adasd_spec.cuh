@@ -368,10 +368,19 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         // ITER so that every warp of every CTA gets ITER - 1 or ITER iterations.
         const int g = rank * kSW + warp;
         const int nwi = (cu1 - cu0 + 31) >> 5;                     // warp-iterations of this CTA
+        // The I_rem warps with one iteration more are taken first among warps 2, 3, 6, 7: warps are
+        // spread over the SM's four schedulers by index modulo 4, and with the two service warps
+        // last, schedulers 2 and 3 carry two compute warps, schedulers 0 and 1 three.
         const int I_lo = nwi / kSW, I_rem = nwi % kSW;
-        const int I_w = min(ITER, I_lo + (warp < I_rem ? 1 : 0));
+        auto extra = [&](int w) -> int {          // 1 if warp w has I_lo + 1 iterations
+            const int light = (w & 3) >> 1;       // 1: its scheduler carries two compute warps
+            const int among = light ? (((w >> 2) << 1) | (w & 1)) : (4 + ((w >> 2) << 1) + (w & 1));
+            return among < I_rem ? 1 : 0;
+        };
+        int wi0 = 0;
+        for (int w = 0; w < warp; ++w) wi0 += I_lo + extra(w);
+        const int I_w = min(ITER, I_lo + extra(warp));
         const bool full = (I_w == ITER);                           // the last iteration exists
-        const int wi0 = warp * I_lo + min(warp, I_rem);
         const int wu0 = cu0 + 32 * wi0;
         const int nwu = max(0, min(32 * I_w, cu1 - wu0));          // units of this warp (last one ragged)
         const uint32_t row_bytes = (uint32_t)nwu * 16u;            // this warp's share of one row
