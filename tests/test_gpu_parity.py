@@ -368,3 +368,89 @@ def test_repeatable_bitwise(torch, adasd):
     for k in res[0]:
         a, b = res[0][k], res[1][k]
         assert torch.equal(a.view(torch.int32), b.view(torch.int32)), k
+
+
+# ------------------------------------------------------------------ CUDA graph replay
+
+def test_adaptive_round_in_a_cuda_graph_replays_like_eager_calls(torch, adasd):
+    """One whole adaptive round (inputs of the round the device counter names, draft steps
+    with the stop check, verification with the fused threshold update) is captured ONCE in a
+    CUDA graph; replaying it R times must leave the sequences in exactly the state that the
+    same R rounds issued call by call leave them in: the hot calls launch from device-resident
+    state only, with nothing decided on the host in between."""
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    # 8200 bf16 logits take the streaming kernels; windows of up to 6 from the stop check
+    wl = synth.WORKLOADS["C5"].scaled(name="graph", B=24, K=6, V=8200, rounds=12)
+    B, K, V, R = wl.B, wl.K, wl.V, 12
+
+    def build():
+        ctx = adasd.Context(B, V, K, dtype=wl.dtype, list_capacity=256, device=0)
+        gs = synth.GpuSynth(wl, str(dev))
+        f32, i32 = dict(dtype=torch.float32, device=dev), dict(dtype=torch.int32, device=dev)
+        zd = torch.empty((B, K, V), dtype=torch.bfloat16, device=dev)
+        zt = torch.empty((B, K + 1, V), dtype=torch.bfloat16, device=dev)
+        U = gs.new_round_uniforms()
+        ud = torch.empty((K, B), **f32)
+        Hk, tokk = torch.zeros((K, B), **f32), torch.zeros((K, B), **i32)
+        stopk = torch.zeros((K, B), dtype=torch.uint8, device=dev)
+        active = torch.ones(B, dtype=torch.uint8, device=dev)
+        dlen, x = torch.zeros(B, **i32), torch.zeros((B, K), **i32)
+        al, nt = torch.zeros(B, **i32), torch.zeros(B, **i32)
+        acc = torch.zeros((3, B), dtype=torch.int64, device=dev)   # sums of windows, accept_len, tokens
+
+        def one_round():
+            gs.draft_rows(0, zd, use_round_dev=True)
+            gs.target_rows(0, zt, use_round_dev=True)
+            gs.round_uniforms(0, U, use_round_dev=True)
+            ud.copy_(U["draft"].T)
+            dlen.zero_()
+            active.fill_(1)
+            for k in range(K):
+                ctx.draft_entropy(zd[:, k, :], Hk[k], u=ud[k], token_out=tokk[k], active=active,
+                                  stop_out=stopk[k], draft_len=dlen, row_stride=K * V)
+            x.copy_(tokk.T)
+            ctx.verify(zd, zt, x, U["target"], U["accept"], al, nt, draft_len=dlen, fuse_update=True)
+            acc[0] += dlen
+            acc[1] += al
+            acc[2] += nt
+            gs.advance_round(1)
+
+        def state():
+            torch.cuda.synchronize()
+            T, nE, nA, nR = ctx.get_thresholds()
+            torch.cuda.synchronize()
+            return dict(T=T.cpu(), nE=nE.cpu(), nA=nA.cpu(), nR=nR.cpu(), acc=acc.cpu(), al=al.cpu(),
+                        nt=nt.cpu(), dlen=dlen.cpu(), status=ctx.status(), round=int(gs.round_dev.item()))
+        return ctx, gs, one_round, state, acc
+
+    # call by call
+    ctx, gs, one_round, state, acc = build()
+    for _ in range(R):
+        one_round()
+    eager = state()
+    ctx.close()
+    assert eager["status"] == 0 and eager["round"] == R
+    assert int(eager["nE"].sum()) > 0 and len(set(eager["dlen"].tolist())) >= 2   # rejections and stops happened
+
+    # captured once, replayed R times
+    ctx, gs, one_round, state, acc = build()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        one_round()                              # untimed first pass outside the capture
+        torch.cuda.synchronize()
+        ctx.reset()
+        gs.round_dev.zero_()
+        acc.zero_()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            one_round()
+        for _ in range(R):
+            g.replay()
+        torch.cuda.synchronize()
+    replayed = state()
+    ctx.close()
+    assert replayed["status"] == 0 and replayed["round"] == R
+    for key in ("T", "nE", "nA", "nR", "acc", "al", "nt", "dlen"):
+        assert torch.equal(eager[key], replayed[key]), key
