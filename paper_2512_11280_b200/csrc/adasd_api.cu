@@ -207,8 +207,10 @@ void fast_setup(adasd_ctx* c, size_t smem_optin) {
     const int V = c->cfg.V;
     if (c->cfg.dtype == ADASD_BF16 && (V & 7) == 0 && V >= 8192 &&
         (V >> 3) <= kDMaxP * kDW * kDMaxChunks * kDChunkUnits) {
-        if (cudaFuncSetAttribute(draft_stream_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kDW * 2 * kDChunkBytes) == cudaSuccess)
+        if (cudaFuncSetAttribute(draft_stream_kernel<kDW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kDW * 2 * kDChunkBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(draft_stream_kernel<kDWBig>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kDWBig * 2 * kDChunkBytes) == cudaSuccess)
             c->draft_stream = true;
         else
             cudaGetLastError();
@@ -492,11 +494,14 @@ int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stri
     cudaStream_t st = (cudaStream_t)stream;
     if (vec && ctx->draft_stream) {
         const int P = draft_stream_p(ctx);
+        // a grid of at most one CTA per SM runs 16 warps per CTA, a larger one 8 (two CTAs per SM)
+        const bool big = (long long)p.B * P <= ctx->sm_count && P * kDWBig <= kDMaxEntries;
+        const int W = big ? kDWBig : kDW;
         cudaLaunchConfig_t lc;
         memset(&lc, 0, sizeof(lc));
         lc.gridDim = dim3((unsigned)(p.B * P), 1, 1);
-        lc.blockDim = dim3(kDThreads, 1, 1);
-        lc.dynamicSmemBytes = (size_t)(kDW * 2 * kDChunkBytes);
+        lc.blockDim = dim3((unsigned)(W * 32), 1, 1);
+        lc.dynamicSmemBytes = (size_t)(W * 2 * kDChunkBytes);
         lc.stream = st;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -505,7 +510,11 @@ int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stri
         attr[0].val.clusterDim.z = 1;
         lc.attrs = attr;
         lc.numAttrs = 1;
-        CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<0>, p));
+        if (big) {
+            CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDWBig>, p));
+        } else {
+            CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDW>, p));
+        }
         return ADASD_OK;
     }
     if (ctx->cfg.dtype == ADASD_BF16)

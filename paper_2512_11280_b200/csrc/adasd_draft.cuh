@@ -17,24 +17,29 @@
 
 namespace adasd {
 
-constexpr int kDW = 8;                         // warps per CTA
-constexpr int kDThreads = kDW * 32;
+constexpr int kDW = 8;                         // warps per CTA when two CTAs share an SM
+constexpr int kDWBig = 16;                     // warps per CTA when the grid has one CTA per SM at most
 constexpr int kDChunkUnits = 256;              // 16-byte units per chunk: 8 iterations of a warp
 constexpr int kDChunkBytes = kDChunkUnits * 16;
 constexpr int kDMaxChunks = 12;                // chunks per warp, at most (V <= 8 * 8 * 12 * 2048)
 constexpr int kDMaxP = 8;
 
+constexpr int kDMaxEntries = 64;               // warps per cluster (P * NW), at most: two table entries per lane
+template <int NW>
 struct __align__(16) DraftShared {
-    float cm[kDMaxP][kDW][kDMaxChunks];        // rank 0: shift in force when a chunk was summed
-    float cs[kDMaxP][kDW][kDMaxChunks];        // rank 0: the chunk's sum of 2^t under that shift
-    float4 wpart[kDMaxP][kDW];                 // rank 0: every warp's (M, S, T, flags)
-    unsigned long long bar[kDW][2];
+    float cm[kDMaxEntries][kDMaxChunks];       // rank 0: shift in force when a chunk was summed, by (rank, warp)
+    float cs[kDMaxEntries][kDMaxChunks];       // rank 0: the chunk's sum of 2^t under that shift
+    float4 wpart[kDMaxEntries];                // rank 0: every warp's (M, S, T, flags)
+    unsigned long long bar[NW][2];
 };
 
-template <int DUMMY = 0>
-__global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams p) {
+// NW warps per CTA: 8 (two CTAs per SM) or 16 (one CTA per SM, for grids that do not fill the
+// SMs twice); P * NW <= kDMaxEntries.
+template <int NW>
+__global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kernel(DraftParams p) {
+    constexpr int kDW = NW;                    // (shadows the namespace constant: warps of THIS kernel)
     extern __shared__ __align__(128) unsigned char dyn_smem[];
-    __shared__ DraftShared sh;
+    __shared__ DraftShared<NW> sh;
     cg::cluster_group cluster = cg::this_cluster();
     const int P = (int)cluster.num_blocks();
     const int rank = (int)cluster.block_rank();
@@ -78,9 +83,9 @@ __global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams 
         issue(1);
         // table entries of chunks this warp does not have: no weight
         if (lane >= nch && lane < kDMaxChunks) {
-            DraftShared* r0 = cluster.map_shared_rank(&sh, 0);
-            r0->cm[rank][warp][lane] = kFloorL;
-            r0->cs[rank][warp][lane] = 0.f;
+            DraftShared<NW>* r0 = cluster.map_shared_rank(&sh, 0);
+            r0->cm[rank * kDW + warp][lane] = kFloorL;
+            r0->cs[rank * kDW + warp][lane] = 0.f;
         }
         for (int c = 0; c < nch; ++c) {
             bool ok = alive && mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u);
@@ -135,15 +140,15 @@ __global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams 
             S2 = __fadd2_rn(S2, Sc);
             const float cs = warp_sum(Sc.x + Sc.y);
             if (lane == 0) {
-                DraftShared* r0 = cluster.map_shared_rank(&sh, 0);
-                r0->cm[rank][warp][c] = M;
-                r0->cs[rank][warp][c] = cs;
+                DraftShared<NW>* r0 = cluster.map_shared_rank(&sh, 0);
+                r0->cm[rank * kDW + warp][c] = M;
+                r0->cs[rank * kDW + warp][c] = cs;
             }
         }
         const float Sw = warp_sum(S2.x + S2.y), Tw = warp_sum(T2.x + T2.y);
         bad = __reduce_or_sync(0xFFFFFFFFu, bad);
         if (lane == 0)
-            cluster.map_shared_rank(&sh, 0)->wpart[rank][warp] = make_float4(M, Sw, Tw, __uint_as_float(bad));
+            cluster.map_shared_rank(&sh, 0)->wpart[rank * kDW + warp] = make_float4(M, Sw, Tw, __uint_as_float(bad));
     }
     cluster.sync();        // totals and tables of every CTA are in rank 0's shared memory
     if (!active || rank != 0) return;
@@ -152,7 +157,7 @@ __global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams 
     if (warp == 0) {
         // row totals: lane l holds warp-entry l (and l + 32 when P * 8 > 32)
         const int NE = P * kDW;
-        const float4* wp = &sh.wpart[0][0];
+        const float4* wp = &sh.wpart[0];
         float4 e0 = lane < NE ? wp[lane] : make_float4(kFloorL, 0.f, 0.f, 0.f);
         float4 e1 = lane + 32 < NE ? wp[lane + 32] : make_float4(kFloorL, 0.f, 0.f, 0.f);
         const float Mr = warp_max_f32(fmaxf(e0.x, e1.x));
@@ -198,8 +203,8 @@ __global__ void __launch_bounds__(kDThreads, 2) draft_stream_kernel(DraftParams 
             if (ent >= 0) {
                 const float ebase = ent < 32 ? __shfl_sync(0xFFFFFFFFu, i0 - w0, ent)
                                              : __shfl_sync(0xFFFFFFFFu, i1 - w1, ent - 32);
-                const float* cmf = &sh.cm[0][0][0] + ent * kDMaxChunks;
-                const float* csf = &sh.cs[0][0][0] + ent * kDMaxChunks;
+                const float* cmf = &sh.cm[0][0] + ent * kDMaxChunks;
+                const float* csf = &sh.cs[0][0] + ent * kDMaxChunks;
                 const float v = lane < kDMaxChunks ? ex2(cmf[lane] - Mr) * csf[lane] : 0.f;
                 float incl = v;
 #pragma unroll
