@@ -76,6 +76,9 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
         }
     };
     float M = kFloorL;                                   // running shift (log2 domain)
+    // the largest logit so far (0 while there is none): t = (z - vM) log2 e is exactly 0 for it,
+    // so that a one-hot row gets S = 1, T = 0 and H = 0 exactly
+    float vM = 0.f;
     float2 S2 = make_float2(0.f, 0.f), T2 = S2;          // lane partials under M
     uint32_t bad = 0u;
     if (active) {
@@ -115,15 +118,15 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
             if (vmax == INFINITY) bad = 1u;
             const float Mc = vmax > ADASD_FLOOR_BF ? vmax * kLog2e : kFloorL;
             if (Mc > M) {                                 // raise the shift, rescale what is summed
-                const float d = M - Mc, f = ex2(d);
+                const float d = M > kFloorL ? (vM - vmax) * kLog2e : kFloorL, f = ex2(d);
                 T2.x = f * fmaf(d, S2.x, T2.x);
                 T2.y = f * fmaf(d, S2.y, T2.y);
                 S2.x *= f;
                 S2.y *= f;
                 M = Mc;
+                vM = vmax;
             }
-            const float nm = M > kFloorL ? -M : 0.f;
-            const float2 nm2 = make_float2(nm, nm), L2 = make_float2(kLog2e, kLog2e);
+            const float2 nv2 = make_float2(-vM, -vM), L2 = make_float2(kLog2e, kLog2e);
             float2 Sc = make_float2(0.f, 0.f);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -131,7 +134,7 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float2 z = unpack2(bclamp2(w[j]));
-                    const float2 t = __ffma2_rn(z, L2, nm2);
+                    const float2 t = __fmul2_rn(__fadd2_rn(z, nv2), L2);
                     const float2 e = make_float2(ex2(t.x), ex2(t.y));
                     Sc = __fadd2_rn(Sc, e);
                     T2 = __ffma2_rn(e, t, T2);

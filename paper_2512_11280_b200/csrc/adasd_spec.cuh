@@ -458,12 +458,12 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             else pass_a(std::false_type{}, n, blocking);
         };
 
-        // The warp's shifts and flags from the packed accumulators.  Shifts live in the log2
-        // domain: M = fl(max * log2 e), and every kept value is 2^(z log2 e - M) with ONE
-        // rounding (an FMA), so sums of different warps combine through the exact differences
-        // of their M.  A slice without a finite logit gets M = kFloorL and all-zero values.
+        // The warp's shifts and flags from the packed accumulators.  Every kept value is
+        // 2^((z - max) log2 e) with the share's own largest logit, exactly 1 for that logit;
+        // shares combine in the log2 domain through the differences of M = fl(max * log2 e).
+        // A slice without a finite logit gets M = kFloorL and all-zero values.
         float Mt_w = kFloorL, Md_w = kFloorL;
-        float nmt_w = 0.f, nmd_w = 0.f;           // FMA addends of pass B (-M, or 0 for an empty slice)
+        float nmt_w = 0.f, nmd_w = 0.f;           // addends of pass B (-max, or 0 for an empty slice)
         uint32_t flags_w = 0;
         auto finish_a = [&](bool bonus) {
             const float2 a = unpack2(a_mT), d = unpack2(a_mD);
@@ -474,8 +474,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const bool has_t = vt > ADASD_FLOOR_BF, has_d = vd > ADASD_FLOOR_BF;
             Mt_w = has_t ? vt * kLog2e : kFloorL;
             Md_w = has_d ? vd * kLog2e : kFloorL;
-            nmt_w = has_t ? -Mt_w : 0.f;
-            nmd_w = has_d ? -Md_w : 0.f;
+            nmt_w = has_t ? -vt : 0.f;
+            nmd_w = has_d ? -vd : 0.f;
             flags_w = __reduce_or_sync(0xFFFFFFFFu, bad | (a_df ? 2u : 0u));
             a_mT = a_mD = 0xFF80FF80u;
             a_df = 0u;
@@ -483,13 +483,15 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         };
 
         // 2^t values of one unit: 8 logits (four packed words) relative to the shift in `nm`
-        auto exps = [&](const uint4& W, const float2 nm, float (&e)[8], float2& S, float2& Tq) {
+        // nv = -(largest logit of the share): t = (z - max) log2 e is exactly 0 for the largest
+        // logit, so that a one-hot row gets S = 1, T = 0, p = 1 and H = 0 exactly.
+        auto exps = [&](const uint4& W, const float2 nv, float (&e)[8], float2& S, float2& Tq) {
             const float2 L2 = make_float2(kLog2e, kLog2e);
             const uint32_t w[4] = {W.x, W.y, W.z, W.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const float2 z = unpack2(bclamp2(w[j]));
-                const float2 t = __ffma2_rn(z, L2, nm);
+                const float2 t = __fmul2_rn(__fadd2_rn(z, nv), L2);
                 const float2 v = make_float2(ex2(t.x), ex2(t.y));
                 e[2 * j] = v.x;
                 e[2 * j + 1] = v.y;
@@ -883,7 +885,9 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
 
             // first message per compute warp (lane w): its scale factors; pass C starts on it
             const float ftw = ex2(w0.x - Mt), fdw = ex2(w0.w - Md);
-            const float at = __fdividef(ftw, St), ad = __fdividef(fdw, Sd);
+            // correctly rounded quotients: a one-hot row must get p = 1 exactly, so that two rows
+            // that are one-hot on the same token give p + q = 2 and a divergence of exactly 0
+            const float at = __fdiv_rn(ftw, St), ad = __fdiv_rn(fdw, Sd);
             if (lane < kSW) *reinterpret_cast<float4*>(&sh.wmsg[par][lane]) = make_float4(at, ad, ftw, __int_as_float(act));
             __syncwarp();
             if (lane == 0) mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.scal_bar[par]));

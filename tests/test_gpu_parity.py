@@ -163,8 +163,14 @@ class Case:
                                    self.ua[b].cpu().numpy(), K_t=K_t, update=update)
 
 
-def test_identical_disjoint_and_onehot_rows(torch, adasd):
-    V, K = 1000, 4
+# every crafted case runs on the generic kernels (small or fp32 rows) and on the streaming
+# kernels (bf16 rows of a multiple of 8 logits, at least 8192 of them)
+GENERIC_AND_STREAMING = [(1000, "float32"), (8200, "bfloat16")]
+
+
+@pytest.mark.parametrize("V,dt", GENERIC_AND_STREAMING)
+def test_identical_disjoint_and_onehot_rows(torch, adasd, V, dt):
+    K = 4
     rng = np.random.default_rng(0)
     ninf = -np.inf
     zd = rng.normal(size=(1, K, V)).astype(np.float32) * 2
@@ -177,7 +183,7 @@ def test_identical_disjoint_and_onehot_rows(torch, adasd):
     zd[0, 2, 17] = 5.0
     zt[0, 2, 17] = 7.0
     x = [[3, 600, 17, 5]]
-    c = Case(torch, adasd, zd, zt, x, rng.random((1, K + 1)), np.full((1, K), 0.5))
+    c = Case(torch, adasd, zd, zt, x, rng.random((1, K + 1)), np.full((1, K), 0.5), dtype=getattr(torch, dt))
     r = c.verify()
     st = oracle.SequenceState(capacity=64)
     o = c.oracle_round(0, st)
@@ -199,9 +205,11 @@ def test_identical_disjoint_and_onehot_rows(torch, adasd):
 
 
 def test_entropy_closed_forms_on_device(torch, adasd):
-    for V in (4, 1000, 128256):
-        ctx = adasd.Context(2, V, 1, dtype=adasd.ADASD_FP32, list_capacity=8)
-        z = torch.zeros((2, V), dtype=torch.float32, device="cuda")
+    # fp32 rows take the generic kernel, long bf16 rows the streaming one
+    for V, dt in ((4, "float32"), (1000, "float32"), (128256, "float32"), (8200, "bfloat16"), (128256, "bfloat16")):
+        ctx = adasd.Context(2, V, 1, dtype=adasd.ADASD_FP32 if dt == "float32" else adasd.ADASD_BF16,
+                            list_capacity=8)
+        z = torch.zeros((2, V), dtype=getattr(torch, dt), device="cuda")
         z[1, :] = -float("inf")
         z[1, V // 3] = 2.5                                      # one-hot
         H = torch.zeros(2, device="cuda")
@@ -217,8 +225,9 @@ def test_entropy_closed_forms_on_device(torch, adasd):
         assert int(stop[0]) == 1 and int(stop[1]) == 0           # H > T_G = 0 is strict
 
 
-def test_windows_zero_to_kmax_and_inactive_rows(torch, adasd):
-    V, K, B = 3000, 32, 5
+@pytest.mark.parametrize("V", [3000, 8200])
+def test_windows_zero_to_kmax_and_inactive_rows(torch, adasd, V):
+    K, B = 32, 5
     rng = np.random.default_rng(4)
     zd = rng.normal(size=(B, K, V)).astype(np.float32) * 3
     zt = zd[:, :, :] + rng.normal(size=(B, K, V)).astype(np.float32)
@@ -241,14 +250,16 @@ def test_windows_zero_to_kmax_and_inactive_rows(torch, adasd):
     assert c.ctx.status() == 0
 
 
-def test_nan_and_all_minus_inf_rows_set_status_not_faults(torch, adasd):
-    V, K = 500, 2
+@pytest.mark.parametrize("V,dt", [(500, "float32"), (8200, "bfloat16")])
+def test_nan_and_all_minus_inf_rows_set_status_not_faults(torch, adasd, V, dt):
+    K = 2
     rng = np.random.default_rng(5)
     zd = rng.normal(size=(2, K, V)).astype(np.float32)
     zt = rng.normal(size=(2, K + 1, V)).astype(np.float32)
     zd[0, 1, 100] = np.nan
     zt[1, 0, :] = -np.inf
-    c = Case(torch, adasd, zd, zt, [[1, 2], [3, 4]], rng.random((2, K + 1)), rng.random((2, K)))
+    c = Case(torch, adasd, zd, zt, [[1, 2], [3, 4]], rng.random((2, K + 1)), rng.random((2, K)),
+             dtype=getattr(torch, dt))
     r = c.verify()
     assert np.isnan(r["H_d"][0, 1]) and np.isnan(r["jsd"][0, 1])
     assert np.isnan(r["H_t"][1, 0]) and r["y"][1, 0] == -1
