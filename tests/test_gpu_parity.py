@@ -465,3 +465,55 @@ def test_adaptive_round_in_a_cuda_graph_replays_like_eager_calls(torch, adasd):
     assert replayed["status"] == 0 and replayed["round"] == R
     for key in ("T", "nE", "nA", "nR", "acc", "al", "nt", "dlen"):
         assert torch.equal(eager[key], replayed[key]), key
+
+
+@pytest.mark.parametrize("V,dt", GENERIC_AND_STREAMING)
+def test_vanilla_mode_crafted_rows(torch, adasd, V, dt):
+    """Vanilla speculative sampling on hand-made rows: identical rows accept with alpha = 1 and
+    the bonus row is sampled; a draft token the target gives no mass is rejected and the
+    residual is the target distribution; an ordinary rejection resamples from max(0, p - q);
+    a shorter window takes its own bonus row."""
+    K, B = 3, 4
+    tdt = getattr(torch, dt)
+    rng = np.random.default_rng(11)
+    zd = rng.normal(size=(B, K, V)).astype(np.float32) * 2
+    zt = zd + rng.normal(size=(B, K, V)).astype(np.float32)
+    zt = np.concatenate([zt, rng.normal(size=(B, 1, V)).astype(np.float32) * 2], axis=1)
+    zt[0, :K] = zd[0]                                      # b0: identical rows everywhere
+    zd[1, 0, :] = -np.inf                                  # b1: one-hot rows on different tokens
+    zt[1, 0, :] = -np.inf
+    zd[1, 0, 7] = 1.5
+    zt[1, 0, 40] = -3.0
+    zt[2, 0] = zd[2, 0]                                    # b2: accepted, then an ordinary rejection
+    x = rng.integers(0, V, size=(B, K)).astype(np.int32)
+    x[1, 0] = 7
+    x[2, 1] = 123
+    zd[2, 1, 123] += 8.0                                   # the draft likes its token far more than the target
+    ua = np.full((B, K), 0.5, dtype=np.float32)
+    ua[2, 1] = 0.9999
+    ua[3, 0] = 0.0
+    ur = np.array([0.3, 0.9, 0.37, 0.62], dtype=np.float32)
+    draft_len = [K, K, K, 1]
+    dev = "cuda"
+    ctx = adasd.Context(B, V, K, dtype=adasd.ADASD_FP32 if dt == "float32" else adasd.ADASD_BF16, list_capacity=8)
+    zd_g = torch.tensor(zd).to(tdt).to(dev)
+    zt_g = torch.tensor(zt).to(tdt).to(dev)
+    x_g = torch.tensor(x, device=dev)
+    al = torch.full((B,), -9, dtype=torch.int32, device=dev)
+    nt = torch.full((B,), -9, dtype=torch.int32, device=dev)
+    alpha = torch.full((B, K), float("nan"), dtype=torch.float32, device=dev)
+    ctx.vanilla_verify(zd_g, zt_g, x_g, torch.tensor(ua, device=dev), torch.tensor(ur, device=dev), al, nt,
+                       draft_len=torch.tensor(draft_len, dtype=torch.int32, device=dev), alpha_out=alpha)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    alpha_h = alpha.cpu().numpy()
+    for b in range(B):
+        K_t = draft_len[b]
+        o = oracle.vanilla_round(raw(zd_g[b, :K_t], torch), raw(zt_g[b], torch), x[b, :K_t], ua[b, :K_t], float(ur[b]))
+        assert int(al[b]) == o["accept_len"], (b, int(al[b]), o)
+        assert o["margin"] > 1e-6 and int(nt[b]) == o["next_token"], (b, int(nt[b]), o)
+        n_seen = min(o["accept_len"] + 1, K_t)
+        assert np.allclose(alpha_h[b, :n_seen], o["alpha"][:n_seen], atol=TOL), (b, alpha_h[b], o["alpha"])
+    assert int(al[0]) == K and (alpha_h[0] == 1.0).all()
+    assert int(al[1]) == 0 and alpha_h[1, 0] == 0.0 and int(nt[1]) == 40
+    assert int(al[2]) == 1 and int(al[3]) == 1
