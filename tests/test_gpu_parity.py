@@ -268,8 +268,9 @@ def test_nan_and_all_minus_inf_rows_set_status_not_faults(torch, adasd, V, dt):
     assert c.ctx.status() == 0                                   # reading clears it
 
 
-def test_fused_update_equals_verify_then_update(torch, adasd):
-    wl = synth.WORKLOADS["C3"].scaled(B=6, K=6, V=4096, rounds=30)
+@pytest.mark.parametrize("V", [4096, 8200])      # generic kernel with the CTA-wide tail; streaming kernel with warp tails
+def test_fused_update_equals_verify_then_update(torch, adasd, V):
+    wl = synth.WORKLOADS["C3"].scaled(B=6, K=6, V=V, rounds=30)
     gs = synth.GpuSynth(wl)
     B, K, V = wl.B, wl.K, wl.V
     zd = torch.empty((B, K, V), dtype=torch.bfloat16, device="cuda")
