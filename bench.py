@@ -35,9 +35,9 @@ import synth  # noqa: E402
 METRIC = "verify_logit_rows_per_s"
 UNIT = "rows/s"
 # DRAM bytes of one verify launch (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic
-# byte, from the ncu capture of workload C3 summarised under profiles/ (143.85 MB against
+# byte, from the ncu capture of workload C3 summarised under profiles/ (143.74 MB against
 # 139.54 MB); traffic grows in proportion to the rows read, so other workloads scale by it.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.029
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.030
 
 
 def measured_peak_gbs():
@@ -100,6 +100,17 @@ def step_rows(wl) -> dict:
     """Logit rows read by one step, per call kind (fixed window K)."""
     B, K = wl.B, wl.K
     return {"draft": B * K, "verify": B * (2 * K + 1), "vanilla": B * (2 * K + 1)}
+
+
+def sfu_figures(B: int, K: int, V: int, verify_ms: float, clocks) -> dict:
+    """Special-function (XU) throughput of the verify launch: nominal peak = 148 SMs x 16
+    results per clock x the SM clock sampled during the run (1965 MHz if none was sampled)."""
+    ops = (3 * B * K + B) * V
+    mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    peak = 148 * 16 * mhz * 1e6
+    achieved = ops / (verify_ms * 1e-3)
+    return {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "Tops/s",
+            "frac": achieved / peak, "ops_per_launch": ops}
 
 
 # ------------------------------------------------------------------------------ N ranks
@@ -284,7 +295,9 @@ def run_ours(args) -> dict:
                      "frac_of_8TBs_nominal": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": verify_bytes, "ms_per_launch": verify_ms,
                      "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * verify_bytes,
-                     "traffic_source": "ncu capture of C3, scaled by the rows of this workload"},
+                     "traffic_source": "ncu capture of C3, scaled by the rows of this workload",
+                     # the pipe that ncu shows busiest: 2 ex2 + 1 lg2 per logit pair, 1 ex2 per bonus logit
+                     "special_function_pipe": sfu_figures(B, K, V, verify_ms, clocks)},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = oracle_sample(synth.WORKLOADS[args.workload], args.cpu_seconds)
