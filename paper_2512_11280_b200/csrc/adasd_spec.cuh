@@ -462,7 +462,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         // 2^((z - max) log2 e) with the share's own largest logit, exactly 1 for that logit;
         // shares combine in the log2 domain through the differences of M = fl(max * log2 e).
         // A slice without a finite logit gets M = kFloorL and all-zero values.
-        float Mt_w = kFloorL, Md_w = kFloorL;
         float nmt_w = 0.f, nmd_w = 0.f;           // addends of pass B (-max, or 0 for an empty slice)
         uint32_t flags_w = 0;
         auto finish_a = [&](bool bonus) {
@@ -472,11 +471,10 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const float vd = bonus ? vt : warp_max_f32(fmaxf(d.x, d.y));
             if (vt == INFINITY || vd == INFINITY || !alive) bad = 1u;
             const bool has_t = vt > ADASD_FLOOR_BF, has_d = vd > ADASD_FLOOR_BF;
-            Mt_w = has_t ? vt * kLog2e : kFloorL;
-            Md_w = has_d ? vd * kLog2e : kFloorL;
             nmt_w = has_t ? -vt : 0.f;
             nmd_w = has_d ? -vd : 0.f;
-            flags_w = __reduce_or_sync(0xFFFFFFFFu, bad | (a_df ? 2u : 0u));
+            // bits 4 and 8 (not published): the target / draft share has no finite logit
+            flags_w = __reduce_or_sync(0xFFFFFFFFu, bad | (a_df ? 2u : 0u)) | (has_t ? 0u : 4u) | (has_d ? 0u : 8u);
             a_mT = a_mD = 0xFF80FF80u;
             a_df = 0u;
             a_done = false;
@@ -650,7 +648,10 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
 
         // ---------------------------------- main loop ----------------------------------------
         int n = 0;                 // sequence number of the current position
-        if (pcx(0).pos < total) pass_a_any(pcx(0).bonus != 0, 0, true);
+        if (pcx(0).pos < total) {
+            pass_a_any(pcx(0).bonus != 0, 0, true);
+            finish_a(pcx(0).bonus != 0);
+        }
         while (pcx(n).pos < total) {
             const int par = n & 1;
             const uint32_t ph = (uint32_t)(n >> 1) & 1u;
@@ -658,19 +659,27 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const int npos = pcx(n + 1).pos;
             const bool nbonus = npos < total && pcx(n + 1).bonus != 0;
 
-            finish_a(bonus);
             if (bonus) pass_b(std::true_type{}, n);
             else pass_b(std::false_type{}, n);
             if (lane == 0) {
                 float4* w = reinterpret_cast<float4*>(&sh.wtab[par][warp]);
+                const float Mt_w = (flags_w & 4u) ? kFloorL : -nmt_w * kLog2e;
+                const float Md_w = (flags_w & 8u) ? kFloorL : -nmd_w * kLog2e;
                 w[0] = make_float4(Mt_w, sB[0], sB[1], Md_w);
-                w[1] = make_float4(sB[2], sB[3], __uint_as_float(flags_w), 0.f);
+                w[1] = make_float4(sB[2], sB[3], __uint_as_float(flags_w & 3u), 0.f);
                 mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.entry_bar[par]));
             }
             __syncwarp();
             // while the control warps exchange the totals: maxima of the next position, if it
             // has landed in the other buffer
-            if (npos < total) pass_a_any(nbonus, n + 1, false);
+            bool a_fin = false;        // the next position's shifts are worked out already
+            if (npos < total) {
+                pass_a_any(nbonus, n + 1, false);
+                if (a_done) {          // nothing of position n needs this warp's shifts any more
+                    finish_a(nbonus);
+                    a_fin = true;
+                }
+            }
             wait_cta(&sh.scal_bar[par], ph);
             const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft
 
@@ -762,7 +771,10 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             __syncwarp();
 
             // the next position's maxima, if its copy had not landed during the exchange
-            if (npos < total) pass_a_any(nbonus, n + 1, true);
+            if (npos < total && !a_fin) {
+                pass_a_any(nbonus, n + 1, true);
+                finish_a(nbonus);
+            }
             ++n;
         }
         // a warp that gave up on a copy still waits (bounded) for whatever it had in flight
