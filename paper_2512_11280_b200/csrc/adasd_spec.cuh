@@ -402,8 +402,9 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const bool bonus = c.bonus != 0;
             uint64_t* bar = bar_of(n);
             unsigned char* dst = bufs + (size_t)(n & 1) * (2 * kRowB);
+            // (the copies may complete before the expected byte count is posted: the phase cannot
+            // end before this warp's one arrival, which comes with the count)
             if (lane == 0) mbar_expect_tx(bar, bonus ? row_bytes : 2u * row_bytes);
-            __syncwarp();
             if (lane < (bonus ? 1 : 2))
                 bulk_g2s(dst + lane * kRowB,
                          reinterpret_cast<const unsigned char*>(lane ? c.src_d : c.src_t) + woff, row_bytes, bar);
