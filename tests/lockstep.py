@@ -73,7 +73,8 @@ def _bump(h: dict, k: int) -> None:
 class Lockstep:
     def __init__(self, wl: synth.Workload, follow: Optional[List[int]] = None,
                  cluster_size: int = 0, list_capacity: Optional[int] = None,
-                 min_kde_samples: int = 2, device: int = 0, check_lists_every: int = 16):
+                 min_kde_samples: int = 2, device: int = 0, check_lists_every: int = 16,
+                 kde_bandwidth: int = 0, reject_rule: int = 0):
         import torch
         import paper_2512_11280_b200 as adasd
         self.torch, self.adasd, self.wl = torch, adasd, wl
@@ -82,7 +83,7 @@ class Lockstep:
         cap = list_capacity or max(64, wl.rounds * wl.K + 8)
         self.ctx = adasd.Context(wl.B, wl.V, wl.K, dtype=wl.dtype, list_capacity=cap,
                                  min_kde_samples=min_kde_samples, cluster_size=cluster_size,
-                                 device=device)
+                                 kde_bandwidth=kde_bandwidth, reject_rule=reject_rule, device=device)
         self.gs = synth.GpuSynth(wl, str(self.dev))
         tdt = torch.bfloat16 if wl.dtype == synth.BF16 else torch.float32
         B, K, V = wl.B, wl.K, wl.V
@@ -103,8 +104,10 @@ class Lockstep:
         self.v_next_token = torch.zeros(B, **i32)
         self.alpha = torch.zeros((B, K), **f32)
         self.rec = self.ctx.new_record()
-        self.states = {b: oracle.SequenceState(capacity=cap + K + 8, min_samples=max(2, min_kde_samples))
+        self.states = {b: oracle.SequenceState(capacity=cap + K + 8, min_samples=max(2, min_kde_samples),
+                                               bw_rule=kde_bandwidth, reject_rule=reject_rule)
                        for b in self.follow}
+        self.reject_rule = reject_rule
         self.report = Report()
         self.check_lists_every = check_lists_every
 
@@ -273,8 +276,11 @@ class Lockstep:
                     self.report.err("p_acc_sensitivity", sens)
                     self._close("p_acc", float(rec["p_acc"][b, i]), P, tol=TOL + sens, ctx=c)
                     u = float(u_accept[b, i])
-                    decisions = {u >= P, u >= Plo, u >= Phi}
-                    if x_h[b, i] != o["y"][i] and (abs(u - P) < TOL or len(decisions) > 1):
+                    # the rejection rule in force: Bernoulli (u >= P) or the fixed threshold P < 1/2
+                    cut = u if self.reject_rule == 0 else 0.5
+                    decisions = {cut >= P, cut >= Plo, cut >= Phi} if self.reject_rule == 0 else \
+                                {P < cut, Plo < cut, Phi < cut}
+                    if x_h[b, i] != o["y"][i] and (abs(cut - P) < TOL or len(decisions) > 1):
                         near = True
                 if near:
                     rep.near_threshold += 1

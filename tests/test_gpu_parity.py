@@ -98,6 +98,15 @@ def test_streaming_kernels_at_every_cluster_size(torch, cs):
     assert len(rep.vanilla_accept_hist) >= 2
 
 
+@pytest.mark.parametrize("V", [2048, 8200])
+def test_scott_bandwidth_and_threshold_rejection_rule(torch, V):
+    # the two readings kept behind flags: Scott's bandwidth factor, and rejection when P(A|d) < 1/2
+    # instead of the Bernoulli draw; enough rounds for the KDE lists to matter
+    wl = synth.WORKLOADS["C3"].scaled(name=f"flags{V}", B=4, K=6, V=V, rounds=60, vanilla=False)
+    rep = run_lockstep(wl, kde_bandwidth=1, reject_rule=1, check_lists_every=20)
+    assert rep.n_rejections > 10 and len(rep.accept_hist) >= 2
+
+
 def test_c2_single_stream_adaptive_window(torch):
     wl = synth.WORKLOADS["C2"].scaled(rounds=40)
     rep = run_lockstep(wl)
