@@ -527,3 +527,73 @@ def test_vanilla_mode_crafted_rows(torch, adasd, V, dt):
     assert int(al[0]) == K and (alpha_h[0] == 1.0).all()
     assert int(al[1]) == 0 and alpha_h[1, 0] == 0.0 and int(nt[1]) == 40
     assert int(al[2]) == 1 and int(al[3]) == 1
+
+
+def test_padded_rows_on_the_streaming_path(torch, adasd):
+    """Rows cut out of a wider buffer (row stride V + 24, a gap between sequences; everything
+    still 16-byte aligned) take the streaming kernels with the caller's strides: same results,
+    bit for bit, as the contiguous copy."""
+    wl = synth.WORKLOADS["C3"].scaled(name="padded", B=3, K=4, V=8200, rounds=2)
+    B, K, V = wl.B, wl.K, wl.V
+    gs = synth.GpuSynth(wl)
+    zd = torch.empty((B, K, V), dtype=torch.bfloat16, device="cuda")
+    zt = torch.empty((B, K + 1, V), dtype=torch.bfloat16, device="cuda")
+    gs.draft_rows(0, zd)
+    gs.target_rows(0, zt)
+    wide_d = torch.full((B, K + 1, V + 24), 7.0, dtype=torch.bfloat16, device="cuda")   # one spare row per sequence
+    wide_t = torch.full((B, K + 2, V + 24), 7.0, dtype=torch.bfloat16, device="cuda")
+    pd, pt = wide_d[:, :K, :V], wide_t[:, :K + 1, :V]
+    pd.copy_(zd)
+    pt.copy_(zt)
+    assert pd.stride() == ((K + 1) * (V + 24), V + 24, 1) and not pd.is_contiguous()
+    U = gs.new_round_uniforms()
+    gs.round_uniforms(0, U)
+    out = []
+    for d_, t_ in ((zd, zt), (pd, pt)):
+        ctx = adasd.Context(B, V, K, list_capacity=64)
+        rec = ctx.new_record()
+        i32 = dict(dtype=torch.int32, device="cuda")
+        H = torch.zeros((K, B), device="cuda")
+        tok = torch.zeros((K, B), **i32)
+        for k in range(K):
+            ctx.draft_entropy(d_[:, k, :], H[k], u=U["draft"][:, k].contiguous(), token_out=tok[k])
+        x = tok.T.contiguous()
+        al, nt, val, vnt = (torch.zeros(B, **i32) for _ in range(4))
+        ctx.verify(d_, t_, x, U["target"], U["accept"], al, nt, record=rec)
+        ctx.vanilla_verify(d_, t_, x, U["vanilla_accept"], U["resample"], val, vnt)
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        out.append(dict(H=H, tok=tok, al=al, nt=nt, val=val, vnt=vnt, **{k: v.clone() for k, v in rec.items()}))
+    for k in out[0]:
+        a, b = out[0][k], out[1][k]
+        assert torch.equal(a.view(torch.int32) if a.dtype == torch.float32 else a,
+                           b.view(torch.int32) if b.dtype == torch.float32 else b), k
+    assert (wide_d[:, K, :] == 7.0).all() and (wide_d[:, :, V:] == 7.0).all()        # nothing written around the rows
+
+
+def test_full_lists_set_the_capacity_flag_and_keep_running(torch, adasd):
+    """A list that is full skips the append and raises ADASD_STATUS_CAPACITY; sizes stay at the
+    capacity and later rounds still run."""
+    wl = synth.WORKLOADS["C3"].scaled(name="cap", B=4, K=6, V=8200, rounds=40, vanilla=False)
+    B, K, V = wl.B, wl.K, wl.V
+    cap = 8
+    ctx = adasd.Context(B, V, K, list_capacity=cap)
+    gs = synth.GpuSynth(wl)
+    zd = torch.empty((B, K, V), dtype=torch.bfloat16, device="cuda")
+    zt = torch.empty((B, K + 1, V), dtype=torch.bfloat16, device="cuda")
+    U = gs.new_round_uniforms()
+    i32 = dict(dtype=torch.int32, device="cuda")
+    al, nt = torch.zeros(B, **i32), torch.zeros(B, **i32)
+    x = torch.zeros((B, K), **i32)
+    seen = 0
+    for r in range(wl.rounds):
+        gs.draft_rows(r, zd)
+        gs.target_rows(r, zt)
+        gs.round_uniforms(r, U)
+        ctx.verify(zd, zt, x, U["target"], U["accept"], al, nt, fuse_update=True)
+        seen |= ctx.status()
+        assert 0 <= int(al.min()) and int(al.max()) <= K and 0 <= int(nt.min()) and int(nt.max()) < V
+    T, nE, nA, nR = ctx.get_thresholds()
+    torch.cuda.synchronize()
+    assert seen & adasd.STATUS_CAPACITY and not (seen & ~adasd.STATUS_CAPACITY)
+    assert int(nR.max()) <= cap and int(nA.max()) <= cap and int(nR.max()) == cap
