@@ -65,7 +65,9 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    cluster.sync();        // every CTA of the cluster is running before anyone writes into rank 0
+    // every CTA of the cluster is running before anyone writes into rank 0 (a CTA on its own
+    // writes to itself, and every warp waits on barriers it set up itself)
+    if (P > 1) cluster.sync();
     bool alive = true;
     auto issue = [&](int c) {
         if (lane == 0 && c < nch) {
@@ -153,7 +155,9 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
         if (lane == 0)
             cluster.map_shared_rank(&sh, 0)->wpart[rank * kDW + warp] = make_float4(M, Sw, Tw, __uint_as_float(bad));
     }
-    cluster.sync();        // totals and tables of every CTA are in rank 0's shared memory
+    // totals and tables of every CTA are in rank 0's shared memory
+    if (P > 1) cluster.sync();
+    else __syncthreads();
     if (!active || rank != 0) return;
     // (rank 0 only reads its own shared memory from here on; nobody writes to it any more)
 
