@@ -186,7 +186,7 @@ void fast_setup_mode(adasd_ctx* c, size_t smem_optin) {
         if (iter < 1 || iter > kSMaxIter) continue;
         const int st = fast_static_smem_iter<MODE>(iter);
         if (st < 0) continue;
-        const int smem = kSW * iter * 2048;
+        const int smem = nwi * 2048;      // two position buffers: 512 bytes per row and warp-iteration
         if (smem > (int)smem_optin - st - 1024) continue;
         const int ncl = fast_occupancy_iter<MODE>(iter, cs, smem);
         const int score = ncl * cs;

@@ -10,7 +10,7 @@
 // Values live in the log2 domain: t = z log2 e - M, 2^t kept in registers for the first
 // iterations and, for the rest, parked in the buffer over logits that have been used up.
 //
-//  * 10 COMPUTE warps per CTA do nothing but the passes over their share of a position
+//  * 12 COMPUTE warps per CTA (three per scheduler) do nothing but the passes over their share of a position
 //    (A: maxima and flags; B: 2^t, S = sum 2^t and T = sum 2^t t; C: (p+q) log2 (p+q) in
 //    AdaSD mode, the residual mass max(0, p - q) of a rejected row in vanilla mode), the
 //    refill of their own buffers and, for the one warp that holds it, the inverse-CDF crossing.
@@ -24,6 +24,11 @@
 //    T_G; vanilla: longest accepted prefix) of completed sequences, off everybody's critical
 //    path; AdaSD tails are handed to the idle tail warps of the cluster's other CTAs.
 //
+// The CTA has 16 warps = four warpgroups.  All threads start with 128 registers; the warpgroup
+// of service warps (control, tail and two idle warps) hands registers back with setmaxnreg and
+// the three warpgroups of compute warps take them: 144 registers per compute thread, 80 per
+// service thread.
+//
 // Every wait (buffer filled, partials in, totals in, message ready, sums in, queue) is bounded:
 // a warp whose wait expires sets ADASD_STATUS_TIMEOUT, stops waiting and copying, and walks
 // through the rest of the protocol, so the kernel always ends.
@@ -33,15 +38,15 @@
 
 namespace adasd {
 
-constexpr int kSW = 10;                          // compute warps per CTA
+constexpr int kSW = 12;                          // compute warps per CTA
 constexpr int kSCtl = kSW;                       // warp index of the control warp
 constexpr int kSTail = kSW + 1;                  // warp index of the tail warp
-constexpr int kSThreads = (kSW + 2) * 32;        // 384: leaves 168 registers per thread
-constexpr int kSRegIter = 6;                     // iterations whose 2^t values stay in registers
+constexpr int kSThreads = (kSW + 4) * 32;        // 512: three warpgroups of compute warps, one of service warps
+constexpr int kSRegIter = 5;                     // iterations whose 2^t values stay in registers
 constexpr int kSMaxIter = 10;                    // largest number of iterations per warp and row
 // Iteration k >= kSRegIter parks its 2^t values in the buffer pieces of iterations 2 (k - kSRegIter)
 // and 2 (k - kSRegIter) + 1, which must have been consumed before it: 2 (k - kSRegIter) + 1 < k.
-static_assert(2 * (kSMaxIter - 1 - kSRegIter) + 1 < kSMaxIter - 1, "parked 2^t values would overwrite unread logits");
+static_assert(2 * (kSMaxIter - 1 - kSRegIter) + 1 <= kSMaxIter - 1, "parked 2^t values would overwrite unread logits");
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
 constexpr int kSPosRing = 16;                    // positions the control warp keeps described
 constexpr int kSWorkQ = 16;                      // tail work queue entries per CTA
@@ -350,6 +355,12 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     cluster.sync();   // barriers and positions are set up in every CTA of the cluster
 
+    // 512 threads start with 128 registers each.  The warpgroup of service warps (two of its four
+    // warps have work) gives registers back, the three warpgroups of compute warps take them:
+    // 12 x 32 x 144 + 4 x 32 x 80 = 65536.
+    if (warp < kSW) asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
+    else asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+
     bool alive = true;         // false after a wait expired: this warp stops waiting and copying
     auto expired = [&]() {
         alive = false;
@@ -368,15 +379,9 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         // ITER so that every warp of every CTA gets ITER - 1 or ITER iterations.
         const int g = rank * kSW + warp;
         const int nwi = (cu1 - cu0 + 31) >> 5;                     // warp-iterations of this CTA
-        // The I_rem warps with one iteration more are taken first among warps 2, 3, 6, 7: warps are
-        // spread over the SM's four schedulers by index modulo 4, and with the two service warps
-        // last, schedulers 2 and 3 carry two compute warps, schedulers 0 and 1 three.
+        // the first I_rem warps have one iteration more (every scheduler carries three compute warps)
         const int I_lo = nwi / kSW, I_rem = nwi % kSW;
-        auto extra = [&](int w) -> int {          // 1 if warp w has I_lo + 1 iterations
-            const int light = (w & 3) >> 1;       // 1: its scheduler carries two compute warps
-            const int among = light ? (((w >> 2) << 1) | (w & 1)) : (4 + ((w >> 2) << 1) + (w & 1));
-            return among < I_rem ? 1 : 0;
-        };
+        auto extra = [&](int w) -> int { return w < I_rem ? 1 : 0; };
         int wi0 = 0;
         for (int w = 0; w < warp; ++w) wi0 += I_lo + extra(w);
         const int I_w = min(ITER, I_lo + extra(warp));
@@ -389,8 +394,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         // Two buffers per warp, one position each: [target share | draft share], ITER * 512 bytes
         // per row.  Position n lives in buffer n & 1 and is replaced by position n + 2 as soon as
         // pass C of position n is done, one whole position before it is needed.
-        constexpr int kRowB = ITER * 512;
-        unsigned char* const bufs = dyn_smem + (size_t)warp * (4 * kRowB);
+        const int kRowB = I_w * 512;              // bytes of one row in this warp's buffers
+        unsigned char* const bufs = dyn_smem + (size_t)wi0 * 2048;
         auto buf_of = [&](int n) -> unsigned char* { return bufs + (size_t)(n & 1) * (2 * kRowB) + (size_t)lane * 16; };
         auto bar_of = [&](int n) -> uint64_t* { return reinterpret_cast<uint64_t*>(&sh.bar[warp][n & 1]); };
         auto pcx = [&](int n) -> const PosCtx& { return sh.pc[n & (kSPosRing - 1)]; };
@@ -1002,7 +1007,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             __threadfence_block();
             *reinterpret_cast<volatile int32_t*>(&sh.n_final) = n;
         }
-    } else {
+    } else if (warp == kSTail) {
         // ================================ tail warp =======================================
         // Leader CTA only: finalises every position of the cluster, in order, as soon as its sums
         // are in, and runs the tail of each sequence whose last position that was.
