@@ -113,6 +113,14 @@ def sfu_figures(B: int, K: int, V: int, verify_ms: float, clocks) -> dict:
             "frac": achieved / peak, "ops_per_launch": ops}
 
 
+def vanilla_launches(wl, sm_count: int) -> int:
+    """Kernels one adasd_vanilla_verify call launches: with enough bf16 rows to fill the GPU
+    several times it runs three (log-sum-exps of all rows, accept test, sampling of one
+    position per sequence), else one."""
+    streaming = wl.dtype == synth.BF16 and wl.V % 8 == 0 and wl.V >= 8192
+    return 3 if streaming and wl.B * (2 * wl.K + 1) >= 6 * sm_count else 1
+
+
 # ------------------------------------------------------------------------------ N ranks
 
 def rank_workload(wl, rank: int, sets: int):
@@ -288,7 +296,7 @@ def run_ours(args) -> dict:
         "e2e": {"value": whole_job_rate(world, rows_step, e2e_steps, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": h_out.numel() * 4,
                 "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": args.steps * (K + 2),
+        "gpu_launches": args.steps * (K + 1 + vanilla_launches(wl, torch.cuda.get_device_properties(dev).multi_processor_count)),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "adasd_verify", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",

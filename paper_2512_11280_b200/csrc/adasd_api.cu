@@ -14,6 +14,7 @@
 #include "adasd_cluster.cuh"
 #include "adasd_spec.cuh"
 #include "adasd_draft.cuh"
+#include "adasd_vanilla.cuh"
 
 using namespace adasd;
 
@@ -32,6 +33,7 @@ struct adasd_ctx {
         ClusterGeom geom;
     } fast[2];
     bool draft_stream;        // the streaming draft kernel is usable for this V / dtype
+    bool lse_stream;          // ... and so is the row log-sum-exp kernel of the vanilla mode
 };
 
 namespace {
@@ -204,6 +206,7 @@ void fast_setup(adasd_ctx* c, size_t smem_optin) {
     fast_setup_mode<MODE_VANILLA>(c, smem_optin);
     // streaming draft kernel: bf16 rows of a multiple of 8 logits, two 4 KB buffers per warp
     c->draft_stream = false;
+    c->lse_stream = false;
     const int V = c->cfg.V;
     if (c->cfg.dtype == ADASD_BF16 && (V & 7) == 0 && V >= 8192 &&
         (V >> 3) <= kDMaxP * kDW * kDMaxChunks * kDChunkUnits) {
@@ -212,6 +215,11 @@ void fast_setup(adasd_ctx* c, size_t smem_optin) {
             cudaFuncSetAttribute(draft_stream_kernel<kDWBig>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kDWBig * 2 * kDChunkBytes) == cudaSuccess)
             c->draft_stream = true;
+        else
+            cudaGetLastError();
+        if (cudaFuncSetAttribute(row_lse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kLW * 2 * kLChunkBytes) == cudaSuccess)
+            c->lse_stream = true;
         else
             cudaGetLastError();
     }
@@ -233,7 +241,8 @@ int draft_stream_p(const adasd_ctx* c) {
 
 template <int ITER, int MODE>
 int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
-    const long long positions = (long long)p.B * (p.Kmax + 1);
+    // positions that will be worked on: all of them, or one per sequence
+    const long long positions = p.only_pos ? (long long)p.B : (long long)p.B * (p.Kmax + 1);
     const adasd_ctx::Fast& f = c->fast[MODE];
     ClusterGeom gq = f.geom;
     if (positions < gq.ncl) gq.ncl = (int)positions;
@@ -301,7 +310,38 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
     const int cs = pick_cluster(ctx, positions);
     const bool vec = vec_ok(p.zd, ctx->cfg.dtype, {p.d_seq, p.d_row}) &&
                      vec_ok(p.zt, ctx->cfg.dtype, {p.t_seq, p.t_row});
-    if (vec && ctx->fast[MODE].iter > 0) return fast_launch_iter<MODE>(ctx, p, stream);
+    if (vec && ctx->fast[MODE].iter > 0) {
+        // Vanilla mode with enough rows to fill the GPU: log-sum-exps of all rows in one light
+        // streaming pass, the accept test per sequence, then the sampling of one position per
+        // sequence.  With fewer rows (less than three per CTA slot of the streaming pass) the
+        // extra launches cost more than they save: everything in the one cluster kernel.
+        const long long rows = (long long)p.B * (2 * p.Kmax + 1);
+        if (MODE == MODE_VANILLA && ctx->lse_stream && rows >= 6LL * ctx->sm_count) {
+            LseParams lp;
+            memset(&lp, 0, sizeof(lp));
+            lp.zd = p.zd;
+            lp.zt = p.zt;
+            lp.d_seq = p.d_seq;
+            lp.d_row = p.d_row;
+            lp.t_seq = p.t_seq;
+            lp.t_row = p.t_row;
+            lp.draft_len = p.draft_len;
+            lp.lse_d = p.sc.lse_d;
+            lp.lse_t = p.sc.lse_t;
+            lp.status = p.st.status;
+            lp.B = p.B;
+            lp.V = p.V;
+            lp.Kmax = p.Kmax;
+            row_lse_kernel<<<2 * ctx->sm_count, kLW * 32, kLW * 2 * kLChunkBytes, stream>>>(lp);
+            CUDA_TRY(cudaGetLastError());
+            vanilla_accept_kernel<<<(p.B + 127) / 128, 128, 0, stream>>>(p, p.sc.only_pos);
+            CUDA_TRY(cudaGetLastError());
+            VerifyParams q = p;
+            q.only_pos = p.sc.only_pos;
+            return fast_launch_iter<MODE>(ctx, q, stream);
+        }
+        return fast_launch_iter<MODE>(ctx, p, stream);
+    }
     if (ctx->cfg.dtype == ADASD_BF16) {
         return vec ? launch_cluster(verify_kernel<__nv_bfloat16, true, MODE>, p, positions, cs, stream)
                    : launch_cluster(verify_kernel<__nv_bfloat16, false, MODE>, p, positions, cs, stream);
@@ -434,6 +474,7 @@ int adasd_create(adasd_ctx** out, const adasd_config* cfg) {
     ALLOC(t.van_flag, B * K);
     ALLOC(t.van_tok, B * (K + 1));
     ALLOC(t.ticket, B);
+    ALLOC(t.only_pos, B);
 #undef ALLOC
     if (rc == ADASD_OK) fast_setup(c, prop.sharedMemPerBlockOptin);
     if (rc == ADASD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ADASD_ERR_CUDA;

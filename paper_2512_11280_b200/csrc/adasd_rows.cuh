@@ -24,6 +24,7 @@ struct Scratch {            // context-owned per-round scratch, all [B,Kmax(+1)]
     int32_t* van_flag;      // [B,Kmax] vanilla: 1 accept / 0 reject
     int32_t* van_tok;       // [B,Kmax+1] vanilla: resample (or bonus) candidate
     uint32_t* ticket;       // [B] arrival counter of a sequence's positions
+    int32_t* only_pos;      // [B] vanilla: the position that is sampled (first rejection or bonus row)
 };
 
 struct VerifyParams {
@@ -38,6 +39,7 @@ struct VerifyParams {
     int32_t* accept_len;
     int32_t* next_token;
     float* alpha_out;
+    const int32_t* only_pos;   // vanilla, streaming path: the one position of each sequence still to be sampled (else null)
     adasd_round_record user;   // caller's record (entries may be null)
     Scratch sc;
     State st;

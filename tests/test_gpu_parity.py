@@ -107,6 +107,15 @@ def test_scott_bandwidth_and_threshold_rejection_rule(torch, V):
     assert rep.n_rejections > 10 and len(rep.accept_hist) >= 2
 
 
+def test_vanilla_mode_with_many_rows_takes_the_three_step_path(torch):
+    # enough rows to fill the GPU several times over: log-sum-exps of all rows in a streaming
+    # pass, the accept test per sequence, then the sampling of one position per sequence
+    wl = synth.WORKLOADS["C3"].scaled(name="manyrows", B=192, K=3, V=8200, rounds=6)
+    assert wl.B * (2 * wl.K + 1) >= 6 * 148
+    rep = run_lockstep(wl, follow=[0, 5, 77, 130, 191], min_kde_samples=3)
+    assert len(rep.vanilla_accept_hist) >= 3
+
+
 def test_c2_single_stream_adaptive_window(torch):
     wl = synth.WORKLOADS["C2"].scaled(rounds=40)
     rep = run_lockstep(wl)
@@ -477,8 +486,10 @@ def test_adaptive_round_in_a_cuda_graph_replays_like_eager_calls(torch, adasd):
         assert torch.equal(eager[key], replayed[key]), key
 
 
-@pytest.mark.parametrize("V,dt", GENERIC_AND_STREAMING)
-def test_vanilla_mode_crafted_rows(torch, adasd, V, dt):
+# the third case repeats the four sequences 56 times: 224 * 7 rows are enough for the three-step
+# path (streaming log-sum-exps, accept test, sampling of one position per sequence)
+@pytest.mark.parametrize("V,dt,tile", [(1000, "float32", 1), (8200, "bfloat16", 1), (8200, "bfloat16", 56)])
+def test_vanilla_mode_crafted_rows(torch, adasd, V, dt, tile):
     """Vanilla speculative sampling on hand-made rows: identical rows accept with alpha = 1 and
     the bonus row is sampled; a draft token the target gives no mass is rejected and the
     residual is the target distribution; an ordinary rejection resamples from max(0, p - q);
@@ -503,7 +514,9 @@ def test_vanilla_mode_crafted_rows(torch, adasd, V, dt):
     ua[2, 1] = 0.9999
     ua[3, 0] = 0.0
     ur = np.array([0.3, 0.9, 0.37, 0.62], dtype=np.float32)
-    draft_len = [K, K, K, 1]
+    draft_len = [K, K, K, 1] * tile
+    zd, zt, x, ua, ur = (np.concatenate([a] * tile, axis=0) for a in (zd, zt, x, ua, ur))
+    B = B * tile
     dev = "cuda"
     ctx = adasd.Context(B, V, K, dtype=adasd.ADASD_FP32 if dt == "float32" else adasd.ADASD_BF16, list_capacity=8)
     zd_g = torch.tensor(zd).to(tdt).to(dev)
@@ -517,7 +530,7 @@ def test_vanilla_mode_crafted_rows(torch, adasd, V, dt):
     torch.cuda.synchronize()
     assert ctx.status() == 0
     alpha_h = alpha.cpu().numpy()
-    for b in range(B):
+    for b in sorted(set(range(4)) | set(range(B - 4, B))):
         K_t = draft_len[b]
         o = oracle.vanilla_round(raw(zd_g[b, :K_t], torch), raw(zt_g[b], torch), x[b, :K_t], ua[b, :K_t], float(ur[b]))
         assert int(al[b]) == o["accept_len"], (b, int(al[b]), o)
@@ -527,6 +540,40 @@ def test_vanilla_mode_crafted_rows(torch, adasd, V, dt):
     assert int(al[0]) == K and (alpha_h[0] == 1.0).all()
     assert int(al[1]) == 0 and alpha_h[1, 0] == 0.0 and int(nt[1]) == 40
     assert int(al[2]) == 1 and int(al[3]) == 1
+    # every copy of a sequence gets the same answers
+    assert torch.equal(al.view(tile, 4), al[:4].expand(tile, 4)) and torch.equal(nt.view(tile, 4), nt[:4].expand(tile, 4))
+
+
+def test_vanilla_three_step_path_flags_nan_and_empty_rows(torch, adasd):
+    """NaN in a draft row and a target row without a finite logit, among enough rows for the
+    three-step path: the position counts as rejected, its alpha is NaN, no token is drawn (-1),
+    the status flag is raised, and every other sequence is unaffected."""
+    V, K, B = 8200, 3, 224
+    rng = np.random.default_rng(21)
+    zd = rng.normal(size=(B, K, V)).astype(np.float32) * 2
+    zt = np.concatenate([zd + rng.normal(size=(B, K, V)).astype(np.float32),
+                         rng.normal(size=(B, 1, V)).astype(np.float32)], axis=1)
+    zt[:, :K] = zd                                         # identical rows: everything is accepted ...
+    zd[17, 1, 4000] = np.nan                               # ... except where a row is unusable
+    zt[200, 0, :] = -np.inf
+    dev = "cuda"
+    ctx = adasd.Context(B, V, K, list_capacity=8)
+    zd_g = torch.tensor(zd).to(torch.bfloat16).to(dev)
+    zt_g = torch.tensor(zt).to(torch.bfloat16).to(dev)
+    x = torch.tensor(rng.integers(0, V, size=(B, K)).astype(np.int32), device=dev)
+    ua = torch.full((B, K), 0.5, device=dev)
+    ur = torch.full((B,), 0.25, device=dev)
+    al = torch.full((B,), -9, dtype=torch.int32, device=dev)
+    nt = torch.full((B,), -9, dtype=torch.int32, device=dev)
+    alpha = torch.zeros((B, K), device=dev)
+    ctx.vanilla_verify(zd_g, zt_g, x, ua, ur, al, nt, alpha_out=alpha)
+    torch.cuda.synchronize()
+    assert ctx.status() == adasd.STATUS_NAN
+    assert int(al[17]) == 1 and int(nt[17]) == -1 and torch.isnan(alpha[17, 1]) and float(alpha[17, 0]) == 1.0
+    assert int(al[200]) == 0 and int(nt[200]) == -1 and torch.isnan(alpha[200, 0])
+    ok = torch.ones(B, dtype=torch.bool, device=dev)
+    ok[17] = ok[200] = False
+    assert (al[ok] == K).all() and (nt[ok] >= 0).all() and (nt[ok] < V).all() and (alpha[ok] == 1.0).all()
 
 
 def test_padded_rows_on_the_streaming_path(torch, adasd):
