@@ -334,7 +334,7 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
             lp.Kmax = p.Kmax;
             row_lse_kernel<<<2 * ctx->sm_count, kLW * 32, kLW * 2 * kLChunkBytes, stream>>>(lp);
             CUDA_TRY(cudaGetLastError());
-            vanilla_accept_kernel<<<(p.B + 127) / 128, 128, 0, stream>>>(p, p.sc.only_pos);
+            vanilla_accept_kernel<<<(p.B + 3) / 4, 128, 0, stream>>>(p, p.sc.only_pos);     // one warp per sequence
             CUDA_TRY(cudaGetLastError());
             VerifyParams q = p;
             q.only_pos = p.sc.only_pos;

@@ -7,7 +7,7 @@
 //
 //  1. row_lse_kernel streams every row of the round once (one `ex2` per logit, no second pass,
 //     nothing kept) and leaves lse_t, lse_d;
-//  2. vanilla_accept_kernel (one thread per sequence) forms the alphas, finds the first rejection
+//  2. vanilla_accept_kernel (one warp per sequence) forms the alphas, finds the first rejection
 //     and names the one position that still needs work;
 //  3. the warp-specialised verification kernel runs in vanilla mode over just those positions
 //     (it reads their row pairs a second time: B row pairs out of B (2K + 1) rows).
@@ -184,45 +184,54 @@ __global__ void __launch_bounds__(kLW * 32, 2) row_lse_kernel(LseParams p) {
     }
 }
 
-// One thread per sequence: alpha_i = min(1, p_i(x_i) / q_i(x_i)) from the log-sum-exps, the
-// accept flags, the accepted length, and the one position whose rows the sampling kernel still
-// has to read (the first rejected one, or the bonus row).  A row with NaN or no finite logit
-// has lse = NaN: it counts as rejected and raises the status flag.
+// One warp per sequence, lane i on candidate i: alpha_i = min(1, p_i(x_i) / q_i(x_i)) from the
+// log-sum-exps, the accept flags, the accepted length, and the one position whose rows the
+// sampling kernel still has to read (the first rejected one, or the bonus row).  A row with NaN
+// or no finite logit has lse = NaN: it counts as rejected and raises the status flag.
 __global__ void vanilla_accept_kernel(VerifyParams p, int32_t* only_pos) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5), i = threadIdx.x & 31;
     if (b >= p.B) return;
     const int K = p.Kmax;
     int kt = p.draft_len ? p.draft_len[b] : K;
     kt = max(0, min(kt, K));
-    const __nv_bfloat16* zt = reinterpret_cast<const __nv_bfloat16*>(p.zt) + (long long)b * p.t_seq;
-    const __nv_bfloat16* zd = reinterpret_cast<const __nv_bfloat16*>(p.zd) + (long long)b * p.d_seq;
-    int w = kt;
-    bool nan_seen = false;
-    for (int i = 0; i < kt; ++i) {
+    bool reject = false, bad = false;
+    if (i < kt) {
         const size_t idd = (size_t)b * K + i;
         const float lt = p.sc.lse_t[(size_t)b * (K + 1) + i], ld = p.sc.lse_d[idd];
-        const bool bad = (lt != lt) || (ld != ld);
+        bad = (lt != lt) || (ld != ld);
         const int xi = p.x[idd];
         float alpha = 0.f;
         if (xi >= 0 && xi < p.V) {
             // ln p(x) and ln q(x), -inf logits clamped; their difference is formed before any
             // scaling so that identical rows give exactly 0, alpha exactly 1
+            const __nv_bfloat16* zt = reinterpret_cast<const __nv_bfloat16*>(p.zt) + (long long)b * p.t_seq;
+            const __nv_bfloat16* zd = reinterpret_cast<const __nv_bfloat16*>(p.zd) + (long long)b * p.d_seq;
             const float lp = fmaxf(__bfloat162float(zt[(long long)i * p.t_row + xi]), ADASD_FLOOR_BF) - lt;
             const float lq = fmaxf(__bfloat162float(zd[(long long)i * p.d_row + xi]), ADASD_FLOOR_BF) - ld;
             alpha = fminf(1.f, ex2(__fmul_rn(__fsub_rn(lp, lq), kLog2e)));
             if (!(ex2(__fmul_rn(lq, kLog2e)) > 0.f)) alpha = 1.f;       // q(x) = 0 cannot have been drafted
         }
         const bool accept = !bad && (p.u_accept[idd] < alpha);
+        reject = !accept;
         p.sc.van_flag[idd] = accept ? 1 : 0;
         if (p.alpha_out) p.alpha_out[idd] = bad ? NAN : alpha;
-        nan_seen |= bad;
-        if (!accept && w == kt) w = i;
+    } else if (i == kt) {
+        const float lb = p.sc.lse_t[(size_t)b * (K + 1) + kt];     // the bonus row
+        bad = (lb != lb);
     }
-    const float lb = p.sc.lse_t[(size_t)b * (K + 1) + kt];     // the bonus row
-    nan_seen |= (lb != lb);
-    if (nan_seen) atomicOr(p.st.status, ADASD_STATUS_NAN);
-    p.accept_len[b] = w;
-    only_pos[b] = w;
+    const unsigned mr = __ballot_sync(0xFFFFFFFFu, reject);
+    const unsigned mb = __ballot_sync(0xFFFFFFFFu, bad);
+    if (i == 0) {
+        // Kmax = 32 leaves no lane for the bonus row: look at it here
+        if (kt == 32) {
+            const float lb = p.sc.lse_t[(size_t)b * (K + 1) + kt];
+            if (lb != lb) atomicOr(p.st.status, ADASD_STATUS_NAN);
+        }
+        if (mb) atomicOr(p.st.status, ADASD_STATUS_NAN);
+        const int w = mr ? (__ffs(mr) - 1) : kt;
+        p.accept_len[b] = w;
+        only_pos[b] = w;
+    }
 }
 
 }  // namespace adasd
