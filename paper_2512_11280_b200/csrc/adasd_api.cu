@@ -34,6 +34,7 @@ struct adasd_ctx {
     } fast[2];
     bool draft_stream;        // the streaming draft kernel is usable for this V / dtype
     bool lse_stream;          // ... and so is the row log-sum-exp kernel of the vanilla mode
+    bool sample_stream;       // ... and its sampling kernel (the vocabulary fits its chunk tables)
 };
 
 namespace {
@@ -207,6 +208,7 @@ void fast_setup(adasd_ctx* c, size_t smem_optin) {
     // streaming draft kernel: bf16 rows of a multiple of 8 logits, two 4 KB buffers per warp
     c->draft_stream = false;
     c->lse_stream = false;
+    c->sample_stream = false;
     const int V = c->cfg.V;
     if (c->cfg.dtype == ADASD_BF16 && (V & 7) == 0 && V >= 8192 &&
         (V >> 3) <= kDMaxP * kDW * kDMaxChunks * kDChunkUnits) {
@@ -222,6 +224,13 @@ void fast_setup(adasd_ctx* c, size_t smem_optin) {
             c->lse_stream = true;
         else
             cudaGetLastError();
+        if (V <= kVMaxV) {
+            if (cudaFuncSetAttribute(vanilla_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kVW * 4 * kVChunkBytes) == cudaSuccess)
+                c->sample_stream = true;
+            else
+                cudaGetLastError();
+        }
     }
 }
 
@@ -241,8 +250,7 @@ int draft_stream_p(const adasd_ctx* c) {
 
 template <int ITER, int MODE>
 int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
-    // positions that will be worked on: all of them, or one per sequence
-    const long long positions = p.only_pos ? (long long)p.B : (long long)p.B * (p.Kmax + 1);
+    const long long positions = (long long)p.B * (p.Kmax + 1);
     const adasd_ctx::Fast& f = c->fast[MODE];
     ClusterGeom gq = f.geom;
     if (positions < gq.ncl) gq.ncl = (int)positions;
@@ -316,7 +324,7 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
         // sequence.  With fewer rows (less than three per CTA slot of the streaming pass) the
         // extra launches cost more than they save: everything in the one cluster kernel.
         const long long rows = (long long)p.B * (2 * p.Kmax + 1);
-        if (MODE == MODE_VANILLA && ctx->lse_stream && rows >= 6LL * ctx->sm_count) {
+        if (MODE == MODE_VANILLA && ctx->lse_stream && ctx->sample_stream && rows >= 6LL * ctx->sm_count) {
             LseParams lp;
             memset(&lp, 0, sizeof(lp));
             lp.zd = p.zd;
@@ -336,9 +344,10 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
             CUDA_TRY(cudaGetLastError());
             vanilla_accept_kernel<<<(p.B + 3) / 4, 128, 0, stream>>>(p, p.sc.only_pos);     // one warp per sequence
             CUDA_TRY(cudaGetLastError());
-            VerifyParams q = p;
-            q.only_pos = p.sc.only_pos;
-            return fast_launch_iter<MODE>(ctx, q, stream);
+            // one CTA per sequence streams the row pair of its one position
+            vanilla_sample_kernel<<<p.B, kVW * 32, kVW * 4 * kVChunkBytes, stream>>>(p, p.sc.only_pos);
+            CUDA_TRY(cudaGetLastError());
+            return ADASD_OK;
         }
         return fast_launch_iter<MODE>(ctx, p, stream);
     }

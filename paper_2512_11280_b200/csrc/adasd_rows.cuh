@@ -39,7 +39,6 @@ struct VerifyParams {
     int32_t* accept_len;
     int32_t* next_token;
     float* alpha_out;
-    const int32_t* only_pos;   // vanilla, streaming path: the one position of each sequence still to be sampled (else null)
     adasd_round_record user;   // caller's record (entries may be null)
     Scratch sc;
     State st;

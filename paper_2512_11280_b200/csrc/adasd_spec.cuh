@@ -311,9 +311,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             if (cl < total) {
                 const int c = (int)cl, b = c / K1;
                 kt = window(b);
-                // (vanilla after the accept kernel: only the position that is sampled)
-                ok = (MODE == MODE_VANILLA && p.only_pos) ? ((c - b * K1) == __ldg(p.only_pos + b))
-                                                          : ((c - b * K1) <= kt);
+                ok = (c - b * K1) <= kt;
             }
             const unsigned m = __ballot_sync(0xFFFFFFFFu, ok);
             if (m) {
@@ -901,8 +899,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     van_accept = u_acc < alpha;
                 }
                 act = bad ? 0 : (bonus ? 1 : (van_accept ? 0 : 2));
-                // the accept kernel has decided already: this position was rejected (or is the bonus row)
-                if (p.only_pos) act = bad ? 0 : (bonus ? 1 : 2);
             }
 
             // first message per compute warp (lane w): its scale factors; pass C starts on it
@@ -1057,7 +1053,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                         tok = -1;
                     }
                     if (MODE == MODE_VANILLA) {
-                        if (!bonus && !p.only_pos) {
+                        if (!bonus) {
                             p.sc.van_flag[idd] = (sh.fin[par][8] != 0.f && !bad) ? 1 : 0;
                             if (p.alpha_out) p.alpha_out[idd] = bad ? NAN : sh.fin[par][7];
                         }
@@ -1093,8 +1089,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     }
                     __threadfence();
                     const unsigned ticket = atomicAdd(p.sc.ticket + b, 1u);
-                    // (one position per sequence when the accept kernel has run)
-                    if (ticket == ((MODE == MODE_VANILLA && p.only_pos) ? 0u : (unsigned)c.kt)) {
+                    if (ticket == (unsigned)c.kt) {
                         p.sc.ticket[b] = 0u;          // ready for the next round
                         done_b = b;
                     }

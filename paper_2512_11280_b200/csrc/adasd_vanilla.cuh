@@ -9,8 +9,10 @@
 //     nothing kept) and leaves lse_t, lse_d;
 //  2. vanilla_accept_kernel (one warp per sequence) forms the alphas, finds the first rejection
 //     and names the one position that still needs work;
-//  3. the warp-specialised verification kernel runs in vanilla mode over just those positions
-//     (it reads their row pairs a second time: B row pairs out of B (2K + 1) rows).
+//  3. vanilla_sample_kernel (one CTA per sequence) streams the row pair of that one position:
+//     with the log-sum-exps known, p and q are final as they are read, so per-chunk sums of the
+//     residual max(0, p - q) locate the chunk of the inverse-CDF crossing, which is scanned again
+//     (B row pairs are read a second time, out of B (2K + 1) rows).
 #pragma once
 
 #include "adasd_cluster.cuh"
@@ -231,6 +233,258 @@ __global__ void vanilla_accept_kernel(VerifyParams p, int32_t* only_pos) {
         const int w = mr ? (__ffs(mr) - 1) : kt;
         p.accept_len[b] = w;
         only_pos[b] = w;
+    }
+}
+
+}  // namespace adasd
+
+namespace adasd {
+
+// ---- step 3 for large batches: the one sampled position of every sequence ------------------
+//
+// With the log-sum-exps known, p = 2^((z_t - lse_t) log2 e) and q likewise are final as they
+// are read: one CTA per sequence streams the row pair once, keeps per-chunk sums of the
+// residual max(0, p - q) (and of p, for the bonus row and for a residual without mass), finds
+// the chunk that holds the inverse-CDF crossing of u and scans just that chunk again.
+constexpr int kVW = 16;                        // warps per CTA
+constexpr int kVChunkUnits = 128;              // 16-byte units per chunk of one row: 4 iterations of a warp
+constexpr int kVChunkBytes = kVChunkUnits * 16;
+constexpr int kVMaxChunks = 16;                // chunks per warp, at most
+
+struct __align__(16) SampleShared {
+    float cr[kVW][kVMaxChunks];                // residual mass of every chunk
+    float cp[kVW][kVMaxChunks];                // target mass of every chunk
+    unsigned long long bar[kVW][2];
+};
+
+// largest V the chunk tables hold
+constexpr int kVMaxV = kVW * kVMaxChunks * kVChunkUnits * 8;
+
+__global__ void __launch_bounds__(kVW * 32, 1) vanilla_sample_kernel(VerifyParams p, const int32_t* only_pos) {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ SampleShared sh;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int b = blockIdx.x;
+    const int K = p.Kmax, K1 = K + 1;
+    int kt = p.draft_len ? __ldg(p.draft_len + b) : K;
+    kt = max(0, min(kt, K));
+    const int i = __ldg(only_pos + b);
+    const bool bonus = (i >= kt);
+    const float lt = p.sc.lse_t[(size_t)b * K1 + i];
+    const float ld = bonus ? 0.f : p.sc.lse_d[(size_t)b * K + i];
+    const bool rowbad = (lt != lt) || (ld != ld);
+
+    const int NU = p.V >> 3;
+    const int wu0 = (int)((long long)warp * NU / kVW), wu1 = (int)((long long)(warp + 1) * NU / kVW);
+    const int nwu = wu1 - wu0;
+    const int nch = min(kVMaxChunks, (nwu + kVChunkUnits - 1) / kVChunkUnits);
+    const unsigned char* const src_t = reinterpret_cast<const unsigned char*>(
+        reinterpret_cast<const __nv_bfloat16*>(p.zt) + (long long)b * p.t_seq + (long long)i * p.t_row) + (size_t)wu0 * 16;
+    const unsigned char* const src_d = reinterpret_cast<const unsigned char*>(
+        reinterpret_cast<const __nv_bfloat16*>(p.zd) + (long long)b * p.d_seq + (long long)min(i, K - 1) * p.d_row) + (size_t)wu0 * 16;
+    unsigned char* const bufs = dyn_smem + (size_t)warp * (4 * kVChunkBytes);   // [buffer][target | draft]
+
+    if (lane == 0) {
+        mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][0]), 1);
+        mbar_init(reinterpret_cast<uint64_t*>(&sh.bar[warp][1]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (lane < kVMaxChunks) {
+        sh.cr[warp][lane] = 0.f;
+        sh.cp[warp][lane] = 0.f;
+    }
+    __syncwarp();
+
+    // weights of one 16-byte unit of both rows: p and max(0, p - q)
+    const float nlt = -lt * kLog2e, nld = -ld * kLog2e;
+    auto weights = [&](const uint4& T, const uint4& D, float (&pv)[8], float (&rv)[8]) {
+        const uint32_t tw[4] = {T.x, T.y, T.z, T.w}, dw[4] = {D.x, D.y, D.z, D.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 zt2 = unpack2(bclamp2(tw[j])), zd2 = unpack2(bclamp2(dw[j]));
+            pv[2 * j] = ex2(fmaf(zt2.x, kLog2e, nlt));
+            pv[2 * j + 1] = ex2(fmaf(zt2.y, kLog2e, nlt));
+            const float q0 = bonus ? 0.f : ex2(fmaf(zd2.x, kLog2e, nld));
+            const float q1 = bonus ? 0.f : ex2(fmaf(zd2.y, kLog2e, nld));
+            rv[2 * j] = fmaxf(pv[2 * j] - q0, 0.f);
+            rv[2 * j + 1] = fmaxf(pv[2 * j + 1] - q1, 0.f);
+        }
+    };
+
+    bool alive = !rowbad;                         // an unusable row is neither copied nor sampled
+    auto issue = [&](int c) {
+        if (alive && lane == 0 && c < nch) {
+            const uint32_t bytes = (uint32_t)min(kVChunkUnits, nwu - c * kVChunkUnits) * 16u;
+            uint64_t* bar = reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]);
+            unsigned char* dst = bufs + (size_t)(c & 1) * (2 * kVChunkBytes);
+            mbar_expect_tx(bar, bonus ? bytes : 2u * bytes);
+            bulk_g2s(dst, src_t + (size_t)c * kVChunkBytes, bytes, bar);
+            if (!bonus) bulk_g2s(dst + kVChunkBytes, src_d + (size_t)c * kVChunkBytes, bytes, bar);
+        }
+    };
+    issue(0);
+    issue(1);
+    const uint4 floor4 = make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
+    int cfail = -1;                               // chunk whose copy never landed
+    for (int c = 0; c < nch && alive; ++c) {
+        bool ok = mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) {
+            if (lane == 0) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+            alive = false;
+            cfail = c;
+            break;
+        }
+        const unsigned char* sb = bufs + (size_t)(c & 1) * (2 * kVChunkBytes) + (size_t)lane * 16;
+        uint4 T[4], D[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool in = c * kVChunkUnits + lane + 32 * k < nwu;
+            T[k] = in ? *reinterpret_cast<const uint4*>(sb + k * 512) : floor4;
+            D[k] = (in && !bonus) ? *reinterpret_cast<const uint4*>(sb + kVChunkBytes + k * 512) : floor4;
+        }
+        __syncwarp();
+        issue(c + 2);                             // the chunk is in registers, its buffer free
+        float ps = 0.f, rs = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float pv[8], rv[8];
+            weights(T[k], D[k], pv, rv);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                ps += pv[j];
+                rs += rv[j];
+            }
+        }
+        ps = warp_sum(ps);
+        rs = warp_sum(rs);
+        if (lane == 0) {
+            sh.cp[warp][c] = ps;
+            sh.cr[warp][c] = rs;
+        }
+    }
+    // a warp that gave up on a copy still waits (bounded) for whatever it had in flight
+    if (cfail >= 0) {
+        for (int c = cfail; c < min(cfail + 2, nch); ++c)
+            mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u);
+    }
+    const int timed_out = __syncthreads_or(cfail >= 0);   // the chunk tables are complete
+    if (warp != 0) return;
+
+    // warp 0: which chunk holds the crossing (index order: warp, chunk), then that chunk again
+    int tok = -1;
+    if (!rowbad && !timed_out) {
+        constexpr int E = kVW * kVMaxChunks;      // 256 table entries, 8 per lane in index order
+        const float* crf = &sh.cr[0][0];
+        const float* cpf = &sh.cp[0][0];
+        float r8[8], p8[8], rl = 0.f, pl = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            r8[j] = crf[lane * 8 + j];
+            p8[j] = cpf[lane * 8 + j];
+            rl += r8[j];
+            pl += p8[j];
+        }
+        const float R = warp_sum(rl), P = warp_sum(pl);
+        const bool use_r = !bonus && R > 0.f;     // a residual without mass: draw from p
+        float w8[8], wl = use_r ? rl : pl;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) w8[j] = use_r ? r8[j] : p8[j];
+        float target = __ldg(p.u_resample + b) * (use_r ? R : P);
+        float incl = wl;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        float run = incl - wl;
+        int hit = -1, last = -1;
+        float hbase = 0.f, lbase = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (w8[j] > 0.f) {
+                last = lane * 8 + j;
+                lbase = run;
+                if (hit < 0 && run + w8[j] > target) {
+                    hit = lane * 8 + j;
+                    hbase = run;
+                }
+            }
+            run += w8[j];
+        }
+        const unsigned mh = __ballot_sync(0xFFFFFFFFu, hit >= 0), ml = __ballot_sync(0xFFFFFFFFu, last >= 0);
+        int ent = -1;
+        float base = 0.f;
+        if (mh) {
+            const int l = __ffs(mh) - 1;
+            ent = __shfl_sync(0xFFFFFFFFu, hit, l);
+            base = __shfl_sync(0xFFFFFFFFu, hbase, l);
+        } else if (ml) {          // rounding left no crossing: last chunk with mass, last token with mass
+            const int l = 31 - __clz(ml);
+            ent = __shfl_sync(0xFFFFFFFFu, last, l);
+            base = __shfl_sync(0xFFFFFFFFu, lbase, l);
+            target = INFINITY;
+        }
+        if (ent >= 0) {
+            const int w = ent / kVMaxChunks, c = ent % kVMaxChunks;
+            const int a0 = (int)((long long)w * NU / kVW), a1 = (int)((long long)(w + 1) * NU / kVW);
+            const int u0 = a0 + c * kVChunkUnits, u1 = min(a1, u0 + kVChunkUnits);
+            const uint4* rowt = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.zt) +
+                                                               (long long)b * p.t_seq + (long long)i * p.t_row);
+            const uint4* rowd = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.zd) +
+                                                               (long long)b * p.d_seq + (long long)min(i, K - 1) * p.d_row);
+            uint4 Tq[4], Dq[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int u = u0 + 32 * k + lane;
+                Tq[k] = u < u1 ? __ldg(rowt + u) : floor4;
+                Dq[k] = (u < u1 && !bonus) ? __ldg(rowd + u) : floor4;
+            }
+            float runw = base;
+            int last_pos = -1;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (tok < 0 && u0 + 32 * k < u1) {          // same for the whole warp
+                    const int u = u0 + 32 * k + lane;
+                    float pv[8], rv[8], wt[8];
+                    weights(Tq[k], Dq[k], pv, rv);
+                    float ls = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        wt[j] = use_r ? rv[j] : pv[j];
+                        ls += wt[j];
+                    }
+                    float li = ls;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const float t = __shfl_up_sync(0xFFFFFFFFu, li, o);
+                        if (lane >= o) li += t;
+                    }
+                    float cc = runw + (li - ls);
+                    int h = -1;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        cc += wt[j];
+                        if (wt[j] > 0.f) {
+                            last_pos = u * 8 + j;
+                            if (h < 0 && cc > target) h = u * 8 + j;
+                        }
+                    }
+                    const unsigned m2 = __ballot_sync(0xFFFFFFFFu, h >= 0);
+                    if (m2) tok = __shfl_sync(0xFFFFFFFFu, h, __ffs(m2) - 1);
+                    runw += __shfl_sync(0xFFFFFFFFu, li, 31);
+                }
+            }
+            if (tok < 0) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xFFFFFFFFu, last_pos, o));
+                tok = last_pos;
+            }
+        }
+    }
+    if (lane == 0) {
+        p.sc.van_tok[(size_t)b * K1 + i] = tok;
+        p.next_token[b] = tok;
     }
 }
 
