@@ -115,10 +115,10 @@ def sfu_figures(B: int, K: int, V: int, verify_ms: float, clocks) -> dict:
 
 def vanilla_launches(wl, sm_count: int) -> int:
     """Kernels one adasd_vanilla_verify call launches: with enough bf16 rows to fill the GPU
-    several times it runs three (log-sum-exps of all rows, accept test, sampling of one
+    it runs three (log-sum-exps of all rows, accept test, sampling of one
     position per sequence), else one."""
     streaming = wl.dtype == synth.BF16 and wl.V % 8 == 0 and wl.V >= 8192
-    return 3 if streaming and wl.B * (2 * wl.K + 1) >= 6 * sm_count else 1
+    return 3 if streaming and wl.B * (2 * wl.K + 1) >= 2 * sm_count else 1
 
 
 # ------------------------------------------------------------------------------ N ranks

@@ -321,10 +321,10 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
     if (vec && ctx->fast[MODE].iter > 0) {
         // Vanilla mode with enough rows to fill the GPU: log-sum-exps of all rows in one light
         // streaming pass, the accept test per sequence, then the sampling of one position per
-        // sequence.  With fewer rows (less than three per CTA slot of the streaming pass) the
-        // extra launches cost more than they save: everything in the one cluster kernel.
+        // sequence.  With fewer rows than CTA slots of the streaming pass: everything in the one
+        // cluster kernel.
         const long long rows = (long long)p.B * (2 * p.Kmax + 1);
-        if (MODE == MODE_VANILLA && ctx->lse_stream && ctx->sample_stream && rows >= 6LL * ctx->sm_count) {
+        if (MODE == MODE_VANILLA && ctx->lse_stream && ctx->sample_stream && rows >= 2LL * ctx->sm_count) {
             LseParams lp;
             memset(&lp, 0, sizeof(lp));
             lp.zd = p.zd;

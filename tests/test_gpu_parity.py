@@ -111,7 +111,7 @@ def test_vanilla_mode_with_many_rows_takes_the_three_step_path(torch):
     # enough rows to fill the GPU several times over: log-sum-exps of all rows in a streaming
     # pass, the accept test per sequence, then the sampling of one position per sequence
     wl = synth.WORKLOADS["C3"].scaled(name="manyrows", B=192, K=3, V=8200, rounds=6)
-    assert wl.B * (2 * wl.K + 1) >= 6 * 148
+    assert wl.B * (2 * wl.K + 1) >= 2 * 148
     rep = run_lockstep(wl, follow=[0, 5, 77, 130, 191], min_kde_samples=3)
     assert len(rep.vanilla_accept_hist) >= 3
 
