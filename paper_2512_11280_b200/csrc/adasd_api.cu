@@ -553,13 +553,17 @@ int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stri
         lc.blockDim = dim3((unsigned)(W * 32), 1, 1);
         lc.dynamicSmemBytes = (size_t)(W * 2 * kDChunkBytes);
         lc.stream = st;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)P;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        // the launch may overlap the tail of the kernel ahead of it (the kernel waits before it
+        // reads anything): draft steps come in runs of short calls
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = attr;
-        lc.numAttrs = 1;
+        lc.numAttrs = 2;
         if (big) {
             CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDWBig>, p));
         } else {

@@ -45,6 +45,10 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
     const int rank = (int)cluster.block_rank();
     const int b = blockIdx.x / P;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // Launched with programmatic stream serialisation: the CTAs may be resident before the
+    // kernel ahead in the stream has finished; nothing it wrote (the logits, the active mask, the
+    // window lengths) is touched before this wait, which returns once that kernel is complete.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const bool active = !(p.active && p.active[b] == 0);      // same in every CTA of the cluster
 
     // this warp's share of the row, in 16-byte units
