@@ -49,6 +49,8 @@ def lib():
         getattr(L, name).restype = _D
     L.oracle_js_distance.argtypes = [_D]
     L.oracle_js_distance.restype = _D
+    L.oracle_js_distance_rows.argtypes = [_P, _P, _I, _P]
+    L.oracle_js_distance_rows.restype = _D
     L.oracle_inv_cdf.argtypes = [_P, _I, _D, _P]
     L.oracle_inv_cdf.restype = _I
     L.oracle_sample_std.argtypes = [_P, _I]
@@ -129,6 +131,14 @@ def jsd_entropy_form(p, q) -> float:
 
 def js_distance(jsd_nats: float) -> float:
     return lib().oracle_js_distance(jsd_nats)
+
+
+def js_distance_rows(p, q) -> tuple:
+    """(d, D_JS in nats) of two distributions, with the exact ends of Sec. 4.4."""
+    p, q = _f64(p), _f64(q)
+    j = C.c_double(0.0)
+    d = lib().oracle_js_distance_rows(p.ctypes.data, q.ctypes.data, p.size, C.byref(j))
+    return d, j.value
 
 
 def inv_cdf(p, u: float) -> tuple:

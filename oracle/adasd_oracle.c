@@ -9,7 +9,8 @@
  * fusion or reordering: sums run left to right in index order.
  *
  * Pins (tests marked "not gpu"): closed forms H(uniform)=ln V, H(one-hot)=0,
- * JSD(p,p)=0, symmetry, JSD<=ln 2 with equality on disjoint supports, equality of
+ * JSD(p,p)=0, symmetry, JSD<=ln 2 with equality on disjoint supports (distance exactly
+ * 1 there, exactly 0 on coinciding rows, whatever the rounding of the sum), equality of
  * the two printed forms of the JS divergence, KL = CE - H, triangle inequality of
  * the JS distance, hand-derived V=4 values, brute-force inverse CDF, Leviathan's
  * output-law identity for the vanilla mode, KDE against quadrature and library
@@ -135,6 +136,39 @@ double oracle_js_distance(double jsd_nats) {
     if (c < 0.0) c = 0.0;
     if (c > ln2) c = ln2;
     return sqrt(c / ln2);
+}
+
+/*
+ * The two ends of the distance (Sec. 4.4: samples whose distance is exactly 0 or 1 stay
+ * out of the KDE lists; the paper meets them where the two distributions coincide or
+ * share no token, as truncated sampling distributions do).  A sum of V rounded terms
+ * cannot be relied on to land on 0 or ln 2 to the last bit, so the ends are decided by
+ * what defines them: p_v = q_v for every v gives D_JS = 0 and d = 0; no v with p_v > 0
+ * and q_v > 0 (disjoint supports) gives D_JS = ln 2 and d = 1.  Every other pair takes
+ * the sum of oracle_jsd and the clamp of oracle_js_distance (which may itself round to
+ * an end).  Returns d and stores D_JS in nats.
+ */
+double oracle_js_distance_rows(const double* p, const double* q, int32_t V, double* jsd_out) {
+    const double ln2 = 0.69314718055994530942;
+    int identical = 1, disjoint = 1;
+    for (int32_t v = 0; v < V; ++v) {
+        if (isnan(p[v]) || isnan(q[v])) {
+            *jsd_out = NAN;
+            return NAN;
+        }
+        if (p[v] != q[v]) identical = 0;
+        if (p[v] > 0.0 && q[v] > 0.0) disjoint = 0;
+    }
+    if (identical) {
+        *jsd_out = 0.0;
+        return 0.0;
+    }
+    if (disjoint) {
+        *jsd_out = ln2;
+        return 1.0;
+    }
+    *jsd_out = oracle_jsd(p, q, V);
+    return oracle_js_distance(*jsd_out);
 }
 
 /*
@@ -272,8 +306,7 @@ static void position_math(const void* zd, const void* zt, int32_t dtype, int32_t
             oracle_widen((const char*)zd + (size_t)i * (size_t)d_row_stride * esz, dtype, V, zz);
             lse_d[i] = oracle_softmax(zz, V, q);
             H_d[i] = oracle_entropy(q, V);
-            jsd[i] = oracle_jsd(p, q, V);
-            dist[i] = oracle_js_distance(jsd[i]);
+            dist[i] = oracle_js_distance_rows(p, q, V, &jsd[i]);
         }
         free(zz);
         free(p);

@@ -126,6 +126,40 @@ def test_jsd_zero_symmetric_bounded():
     assert oracle.js_distance(LN2 + 1e-9) == 1.0 and oracle.js_distance(-1e-12) == 0.0
 
 
+def test_distance_ends_are_exact_whatever_the_rounding_of_the_sum():
+    """Sec. 4.4: d is exactly 0 for coinciding rows and exactly 1 for rows that share no
+    token, also where the float64 sum of V terms misses 0 or ln 2 in its last bits."""
+    r = np.random.default_rng(7)
+    missed = 0
+    for V in (100, 5001, 128256):
+        p = np.zeros(V)
+        q = np.zeros(V)
+        cut = V // 3
+        p[:cut] = r.random(cut) ** 4
+        q[cut:] = r.random(V - cut) ** 4
+        p /= p.sum()
+        q /= q.sum()
+        missed += oracle.jsd(p, q) != LN2            # the plain sum need not hit ln 2
+        d, J = oracle.js_distance_rows(p, q)
+        assert d == 1.0 and J == LN2
+        assert oracle.js_distance_rows(q, p) == (1.0, LN2)
+        d, J = oracle.js_distance_rows(p, p.copy())
+        assert d == 0.0 and J == 0.0
+        # one shared token of tiny mass: no longer disjoint, the sum decides (just below 1)
+        q2 = q.copy()
+        q2[0] = 1e-9
+        q2 /= q2.sum()
+        d, J = oracle.js_distance_rows(p, q2)
+        assert J == oracle.jsd(p, q2) and d == oracle.js_distance(J) and 1.0 - 1e-6 < d <= 1.0
+        # ordinary pair: the plain definitions
+        a, b = rand_dist(V, 0.1), rand_dist(V, 0.1)
+        d, J = oracle.js_distance_rows(a, b)
+        assert J == oracle.jsd(a, b) and d == oracle.js_distance(J) and 0.0 < d < 1.0
+    assert missed > 0, "the case this rule exists for did not occur"
+    d, J = oracle.js_distance_rows([0.5, np.nan], [0.5, 0.5])
+    assert math.isnan(d) and math.isnan(J)
+
+
 def test_jsd_two_printed_forms_agree():
     for V in (4, 333, 20000):
         p, q = rand_dist(V, 0.1), rand_dist(V, 0.1)
