@@ -29,6 +29,11 @@
  *     exhausted, NaN / all -inf rows, a bounded wait that expired) set sticky bits
  *     in a status word read with adasd_status(); the call never traps or hangs.
  *   - A context is bound to one device and must be used from one stream at a time.
+ *     The hot calls launch on the calling thread's current device: when that is not the
+ *     context's device they return ADASD_ERR_DEVICE and launch nothing (create, destroy,
+ *     state_export/import and status switch to the context's device themselves).
+ *   - Conditions only the device can see never become return codes: a NaN row, a full
+ *     list or an expired wait is reported through the status word alone.
  */
 #ifndef ADASD_H
 #define ADASD_H
@@ -42,13 +47,13 @@ extern "C" {
 
 #define ADASD_OK 0
 #define ADASD_ERR_NULL (-1)      /* a required pointer is NULL */
-#define ADASD_ERR_ALIGN (-2)     /* a pointer that must be aligned is not */
+#define ADASD_ERR_ALIGN (-2)     /* a pointer is not aligned to its element type (4 bytes for float /
+                                    int32 arrays, 2 or 4 for logits); nothing is launched */
 #define ADASD_ERR_SHAPE (-3)     /* a size, stride or window is out of range */
 #define ADASD_ERR_DTYPE (-4)     /* unknown dtype / rule */
 #define ADASD_ERR_CAPACITY (-5)  /* size beyond a stated maximum */
-#define ADASD_ERR_TIMEOUT (-6)   /* a bounded device wait expired */
 #define ADASD_ERR_CUDA (-7)      /* a CUDA runtime call failed */
-#define ADASD_ERR_NAN (-8)       /* a row held NaN or no finite logit */
+#define ADASD_ERR_DEVICE (-9)    /* the calling thread's current device is not the context's device */
 
 /* bits of the sticky device status word */
 #define ADASD_STATUS_CAPACITY 1u /* an append was skipped: list full */
@@ -157,6 +162,10 @@ int adasd_verify(adasd_ctx* ctx, const void* draft_logits_dev, const void* targe
  * append lines of step 2 and step 3): accepted d_i with 0 < d_i < 1 go to L_D^A; at a
  * rejection H(q_i) goes to L_E^R and d_i (if 0 < d_i < 1) to L_D^R; T_G = mean(L_E^R).
  * The record must carry H_d, dist, draft_len, accept_len and rejected.
+ * A rejected candidate whose entropy is not finite (its row held NaN or no finite logit;
+ * ADASD_STATUS_NAN is already set) is not recorded, so T_G stays finite.  An append to a
+ * list that already holds list_capacity entries is skipped whole (L_E^R too: T_G stays the
+ * mean of what the list holds) and sets ADASD_STATUS_CAPACITY.
  */
 int adasd_update_thresholds(adasd_ctx* ctx, const adasd_round_record* record, void* stream);
 
@@ -220,7 +229,9 @@ int adasd_get_thresholds(adasd_ctx* ctx, float* T_G_dev, int32_t* nE_dev, int32_
                          int32_t* nR_dev, void* stream);
 
 /*
- * Checkpoint of one sequence's adaptive state to / from HOST memory.  Layout:
+ * Checkpoint of ONE sequence's adaptive state to / from HOST memory (a whole context is
+ * saved sequence by sequence; per-sequence is what resuming or migrating a single request
+ * needs).  Layout:
  *   int32 nE, nA, nR, pad; float T_G, pad; then nE + nA + nR floats (L_E^R, L_D^A, L_D^R).
  * Export: call with host_buf = NULL to get the size in *bytes.  Both synchronise the
  * device.  Import recomputes the running sums from the lists.

@@ -73,6 +73,15 @@ def lib():
     return L
 
 
+def set_threads(n: int) -> None:
+    """OpenMP threads the CALLING thread's oracle calls use from now on (the verify round
+    runs its positions in parallel); lets a harness run several sequences side by side."""
+    L = lib()
+    L.omp_set_num_threads.argtypes = [C.c_int]
+    L.omp_set_num_threads.restype = None
+    L.omp_set_num_threads(max(1, int(n)))
+
+
 def _f64(a) -> np.ndarray:
     return np.ascontiguousarray(a, dtype=np.float64)
 

@@ -73,11 +73,14 @@ double oracle_softmax(const double* z, int32_t V, double* p) {
     return m + log(S);
 }
 
-/* Entropy H(p) = -sum p log p in nats, 0 log 0 := 0 (Appendix A, entropy). */
+/* Entropy H(p) = -sum p log p in nats, 0 log 0 := 0 (Appendix A, entropy).
+ * NaN for the NaN row that oracle_softmax gives an unusable logit row. */
 double oracle_entropy(const double* p, int32_t V) {
     double H = 0.0;
-    for (int32_t v = 0; v < V; ++v)
+    for (int32_t v = 0; v < V; ++v) {
+        if (isnan(p[v])) return NAN;
         if (p[v] > 0.0) H -= p[v] * log(p[v]);
+    }
     return H;
 }
 
@@ -360,11 +363,14 @@ void oracle_verify_round(const void* zd, const void* zt, int32_t dtype, int32_t 
         p_acc[i] = PA;
         int rej = reject_rule == 0 ? ((double)u_accept[i] >= PA) : (PA < 0.5);
         if (x[i] != y[i] && rej) {
-            if (update) {
-                LE[nEw] = H_d[i];                     /* record rejected entropy */
-                if (0.0 < d && d < 1.0) LR[nRw++] = d;
+            /* record rejected entropy; a position one of whose rows holds NaN or no finite
+             * logit has no distance, and nothing of it is recorded (the paper is silent on
+             * such rows: they are rejected and leave the lists, and so T_G, as they were) */
+            if (isfinite(H_d[i]) && !isnan(d)) {
+                if (update) LE[nEw] = H_d[i];
+                nEw++;
             }
-            nEw++;
+            if (update && 0.0 < d && d < 1.0) LR[nRw++] = d;
             w = i;                                    /* w <- i - 1 in 1-based terms */
             broke = 1;
             break;

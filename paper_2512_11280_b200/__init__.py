@@ -5,7 +5,8 @@ marshals arguments (device pointers of torch tensors, strides, streams).  There 
 no CPU fallback: importing works anywhere, but every call needs the built library
 and a CUDA device and raises otherwise.
 """
-from .binding import (ADASD_BF16, ADASD_FP32, ADASD_FUSE_UPDATE, ADASD_KMAX_LIMIT, STATUS_CAPACITY,
+from .binding import (ERR_ALIGN, ERR_CAPACITY, ERR_CUDA, ERR_DEVICE, ERR_DTYPE, ERR_NULL, ERR_SHAPE,
+                      ADASD_BF16, ADASD_FP32, ADASD_FUSE_UPDATE, ADASD_KMAX_LIMIT, STATUS_CAPACITY,
                       STATUS_NAN, STATUS_TIMEOUT, AdasdConfig, AdasdError, Context, RoundRecord,
                       adasd_create, adasd_destroy, adasd_draft_entropy, adasd_get_thresholds,
                       adasd_reset, adasd_state_export, adasd_state_import, adasd_status,

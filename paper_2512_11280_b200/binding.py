@@ -18,6 +18,7 @@ ADASD_BF16, ADASD_FP32 = 0, 1
 ADASD_FUSE_UPDATE = 1
 ADASD_KMAX_LIMIT = 32
 STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_NAN = 1, 2, 4
+ERR_NULL, ERR_ALIGN, ERR_SHAPE, ERR_DTYPE, ERR_CAPACITY, ERR_CUDA, ERR_DEVICE = -1, -2, -3, -4, -5, -7, -9
 
 
 class AdasdError(RuntimeError):

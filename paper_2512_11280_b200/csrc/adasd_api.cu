@@ -59,6 +59,25 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline size_t elt_size(int dtype) { return dtype == ADASD_BF16 ? 2 : 4; }
 
+// NULL counts as aligned: whether a pointer may be NULL is checked where it is used.
+inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline bool aligned4(std::initializer_list<const void*> ps) {
+    for (const void* p : ps)
+        if (!aligned_to(p, 4)) return false;
+    return true;
+}
+
+// The hot calls launch on the calling thread's current device with this context's pointers:
+// refuse when that is another GPU.
+int check_device(const adasd_ctx* c) {
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) {
+        cudaGetLastError();
+        return ADASD_ERR_CUDA;
+    }
+    return cur == c->cfg.device ? ADASD_OK : ADASD_ERR_DEVICE;
+}
+
 // Rows can take 16-byte loads when the base and every stride are 16-byte multiples.
 inline bool vec_ok(const void* base, int dtype, std::initializer_list<long long> strides) {
     if (!aligned16(base)) return false;
@@ -288,6 +307,9 @@ int fill_verify_params(adasd_ctx* ctx, VerifyParams& p, const void* zd, const vo
                        const int32_t* x, const int32_t* draft_len) {
     if (!ctx || !zd || !zt || !x) return ADASD_ERR_NULL;
     int rc;
+    if ((rc = check_device(ctx)) != ADASD_OK) return rc;
+    const size_t es = elt_size(ctx->cfg.dtype);
+    if (!aligned_to(zd, es) || !aligned_to(zt, es) || !aligned4({x, draft_len})) return ADASD_ERR_ALIGN;
     if ((rc = check_strides(ctx, d_seq, d_row)) != ADASD_OK) return rc;
     if ((rc = check_strides(ctx, t_seq, t_row)) != ADASD_OK) return rc;
     memset(&p, 0, sizeof(p));
@@ -509,6 +531,8 @@ int adasd_destroy(adasd_ctx* ctx) {
 
 int adasd_reset(adasd_ctx* ctx, const int32_t* seq_ids_dev, int32_t n, void* stream) {
     if (!ctx) return ADASD_ERR_NULL;
+    if (int rc = check_device(ctx)) return rc;
+    if (!aligned4({seq_ids_dev})) return ADASD_ERR_ALIGN;
     if (!seq_ids_dev) n = ctx->cfg.B;
     if (n < 0) return ADASD_ERR_SHAPE;
     if (n == 0) return ADASD_OK;
@@ -524,6 +548,10 @@ int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stri
                         int32_t* draft_len_inout_dev, void* stream) {
     if (!ctx || !logits_dev || !H_out_dev) return ADASD_ERR_NULL;
     if ((u_dev == nullptr) != (token_out_dev == nullptr)) return ADASD_ERR_NULL;
+    if (int rc = check_device(ctx)) return rc;
+    if (!aligned_to(logits_dev, elt_size(ctx->cfg.dtype)) ||
+        !aligned4({u_dev, H_out_dev, lse_out_dev, token_out_dev, draft_len_inout_dev}))
+        return ADASD_ERR_ALIGN;
     if (row_stride < ctx->cfg.V) return ADASD_ERR_SHAPE;
     DraftParams p;
     memset(&p, 0, sizeof(p));
@@ -591,6 +619,11 @@ int adasd_verify(adasd_ctx* ctx, const void* draft_logits_dev, const void* targe
     if (rc != ADASD_OK) return rc;
     if (!u_target_dev || !u_accept_dev || !accept_len_dev || !next_token_dev)
         return ADASD_ERR_NULL;
+    if (!aligned4({u_target_dev, u_accept_dev, accept_len_dev, next_token_dev})) return ADASD_ERR_ALIGN;
+    if (record && !aligned4({record->H_d, record->H_t, record->lse_d, record->lse_t, record->jsd,
+                             record->dist, record->p_acc, record->y, record->draft_len,
+                             record->accept_len, record->rejected}))
+        return ADASD_ERR_ALIGN;
     if (flags & ~ADASD_FUSE_UPDATE) return ADASD_ERR_SHAPE;
     p.u_target = u_target_dev;
     p.u_accept = u_accept_dev;
@@ -606,6 +639,9 @@ int adasd_update_thresholds(adasd_ctx* ctx, const adasd_round_record* record, vo
     if (!record->H_d || !record->dist || !record->draft_len || !record->accept_len ||
         !record->rejected)
         return ADASD_ERR_NULL;
+    if (int rc = check_device(ctx)) return rc;
+    if (!aligned4({record->H_d, record->dist, record->draft_len, record->accept_len, record->rejected}))
+        return ADASD_ERR_ALIGN;
     const int B = ctx->cfg.B;
     update_kernel<<<(B + 127) / 128, 128, 0, (cudaStream_t)stream>>>(ctx->st, *record, B,
                                                                      ctx->cfg.Kmax);
@@ -627,6 +663,8 @@ int adasd_vanilla_verify(adasd_ctx* ctx, const void* draft_logits_dev,
     if (rc != ADASD_OK) return rc;
     if (!u_accept_dev || !u_resample_dev || !accept_len_dev || !next_token_dev)
         return ADASD_ERR_NULL;
+    if (!aligned4({u_accept_dev, u_resample_dev, accept_len_dev, next_token_dev, alpha_out_dev}))
+        return ADASD_ERR_ALIGN;
     p.u_accept = u_accept_dev;
     p.u_resample = u_resample_dev;
     p.accept_len = accept_len_dev;
@@ -638,6 +676,8 @@ int adasd_vanilla_verify(adasd_ctx* ctx, const void* draft_logits_dev,
 int adasd_get_thresholds(adasd_ctx* ctx, float* T_G_dev, int32_t* nE_dev, int32_t* nA_dev,
                          int32_t* nR_dev, void* stream) {
     if (!ctx) return ADASD_ERR_NULL;
+    if (int rc = check_device(ctx)) return rc;
+    if (!aligned4({T_G_dev, nE_dev, nA_dev, nR_dev})) return ADASD_ERR_ALIGN;
     const int B = ctx->cfg.B;
     get_thresholds_kernel<<<(B + 127) / 128, 128, 0, (cudaStream_t)stream>>>(
         ctx->st, T_G_dev, nE_dev, nA_dev, nR_dev, B);
@@ -752,6 +792,10 @@ int adasd_vanilla_verify_static(int32_t B, int32_t V, int32_t Kmax, int32_t dtyp
         return ADASD_ERR_CAPACITY;
     if (d_row_stride < V || t_row_stride < V || d_seq_stride < 0 || t_seq_stride < 0)
         return ADASD_ERR_SHAPE;
+    if (!aligned_to(draft_logits_dev, elt_size(dtype)) || !aligned_to(target_logits_dev, elt_size(dtype)) ||
+        !aligned4({draft_tokens_dev, draft_len_dev, u_accept_dev, u_resample_dev, accept_len_dev,
+                   next_token_dev, alpha_out_dev, status_out_dev}))
+        return ADASD_ERR_ALIGN;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
         cudaGetLastError();
@@ -814,13 +858,12 @@ const char* adasd_strerror(int code) {
     switch (code) {
         case ADASD_OK: return "ok";
         case ADASD_ERR_NULL: return "a required pointer is NULL";
-        case ADASD_ERR_ALIGN: return "pointer not aligned as required";
+        case ADASD_ERR_ALIGN: return "a pointer is not aligned to its element type";
         case ADASD_ERR_SHAPE: return "size, stride or window out of range";
         case ADASD_ERR_DTYPE: return "unknown dtype or rule";
         case ADASD_ERR_CAPACITY: return "size beyond a stated maximum";
-        case ADASD_ERR_TIMEOUT: return "a bounded device wait expired";
         case ADASD_ERR_CUDA: return "a CUDA runtime call failed";
-        case ADASD_ERR_NAN: return "a row held NaN or no finite logit";
+        case ADASD_ERR_DEVICE: return "the current device is not the context's device";
         default: return "unknown error";
     }
 }

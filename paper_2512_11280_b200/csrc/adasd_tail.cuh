@@ -125,13 +125,24 @@ __device__ __forceinline__ void apply_update(State& st, int b, int w, bool rejec
     st.sumA[b] = sA;
     st.sumA2[b] = sA2;
     if (rejected) {
+        // The entropy of a row with NaN or no finite logit is NaN (the status word says so
+        // already): recording it would leave T_G = NaN and switch the draft-stop check off for
+        // good.  A full list skips the append whole, like the other two lists, so that T_G stays
+        // the mean of the entries the list holds (what a checkpoint restores).
+        const float Hw = H[w];
         int nE = st.nE[b];
-        if (nE < cap) st.LE[(size_t)b * cap + nE] = H[w];
-        double sE = st.sumE[b] + (double)H[w];
-        ++nE;
-        st.nE[b] = nE;
-        st.sumE[b] = sE;
-        st.T_G[b] = (float)(sE / (double)nE);  // T_G <- average(L_E^R)
+        if (Hw == Hw && fabsf(Hw) < INFINITY) {
+            if (nE < cap) {
+                st.LE[(size_t)b * cap + nE] = Hw;
+                double sE = st.sumE[b] + (double)Hw;
+                ++nE;
+                st.nE[b] = nE;
+                st.sumE[b] = sE;
+                st.T_G[b] = (float)(sE / (double)nE);  // T_G <- average(L_E^R)
+            } else {
+                atomicOr(st.status, ADASD_STATUS_CAPACITY);
+            }
+        }
         float dw = d[w];
         if (dw > 0.f && dw < 1.f) {
             int nR = st.nR[b];

@@ -20,6 +20,8 @@ rounds stay comparable.  A disagreement anywhere else raises ParityError.
 from __future__ import annotations
 
 import math
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field
 from typing import List, Optional
 
@@ -46,6 +48,9 @@ class Report:
     near_ties: int = 0
     tie_flips: int = 0
     resyncs: int = 0
+    r6_resyncs: int = 0            # of those: the flagged position was a distance within TOL of 0 or 1
+    p_acc_checked: int = 0         # P(A|d) comparisons made
+    p_acc_beyond_tol: int = 0      # of those: |diff| > TOL, inside the band the steepness of P in d allows
     max_err: dict = field(default_factory=dict)
     accept_hist: dict = field(default_factory=dict)
     window_hist: dict = field(default_factory=dict)
@@ -57,9 +62,12 @@ class Report:
             self.max_err[name] = max(self.max_err.get(name, 0.0), float(e))
 
     def summary(self) -> dict:
-        return dict(rounds=self.rounds, positions=self.positions, draft_rows=self.draft_rows,
-                    near_threshold=self.near_threshold, flips=self.flips, near_ties=self.near_ties,
-                    tie_flips=self.tie_flips, resyncs=self.resyncs, n_rejections=self.n_rejections,
+        counts = dict(rounds=self.rounds, positions=self.positions, draft_rows=self.draft_rows,
+                      near_threshold=self.near_threshold, flips=self.flips, near_ties=self.near_ties,
+                      tie_flips=self.tie_flips, resyncs=self.resyncs, r6_resyncs=self.r6_resyncs,
+                      p_acc_checked=self.p_acc_checked, p_acc_beyond_tol=self.p_acc_beyond_tol,
+                      n_rejections=self.n_rejections)
+        return dict({k: int(v) for k, v in counts.items()},
                     max_err={k: float(f"{v:.3e}") for k, v in self.max_err.items()},
                     accept_hist=dict(sorted(self.accept_hist.items())),
                     window_hist=dict(sorted(self.window_hist.items())),
@@ -110,6 +118,12 @@ class Lockstep:
         self.reject_rule = reject_rule
         self.report = Report()
         self.check_lists_every = check_lists_every
+        # the oracle rounds of the followed sequences run side by side (ctypes releases the GIL);
+        # each worker gives the positions of its verify round its share of the host cores
+        cores = len(os.sched_getaffinity(0))
+        workers = max(1, min(len(self.follow), cores))
+        omp = max(1, cores // workers)
+        self.pool = ThreadPoolExecutor(max_workers=workers, initializer=lambda: oracle.set_threads(omp))
 
     # -------------------------------------------------------------- helpers
     def _up(self, a: np.ndarray):
@@ -145,15 +159,16 @@ class Lockstep:
         # ---- oracle draft phase for the followed sequences (host rows)
         fb = np.array(self.follow, dtype=np.int32)
         hd, ht = synth.host_round(wl, r, fb)
-        o_draft = {}
-        for n, b in enumerate(self.follow):
+        def draft_phase(n):
+            b = self.follow[n]
             st, steps = self.states[b], []
             for k in range(K):
                 d = oracle.draft_step(hd[n, k], float(u_draft[b, k]), st.T_G.value)
                 steps.append(d)
                 if wl.adaptive_window and d["stop"]:
                     break
-            o_draft[b] = steps
+            return steps
+        o_draft = dict(zip(self.follow, self.pool.map(draft_phase, range(len(self.follow)))))
 
         # ---- GPU draft phase
         self.gs.draft_rows(r, self.zd)
@@ -233,16 +248,28 @@ class Lockstep:
         x_h = self.x.cpu().numpy()
         T_dev, nE_dev, nA_dev, nR_dev = (t.cpu().numpy() for t in self.ctx.get_thresholds())
 
-        for n, b in enumerate(self.follow):
+        def verify_phase(n):
+            b = self.follow[n]
             st = self.states[b]
             K_t = len(o_draft[b])
             LA0 = st.LA[: st.nA.value].copy()
             LR0 = st.LR[: st.nR.value].copy()
             o = oracle.verify_round(st, hd[n], ht[n], x_h[b, :K_t], u_target[b], u_accept[b], K_t=K_t)
+            ov = None
+            if wl.vanilla:
+                ov = oracle.vanilla_round(hd[n][:K_t], ht[n], x_h[b, :K_t], u_vacc[b, :K_t], float(u_res[b]))
+            return LA0, LR0, o, ov
+        o_verify = list(self.pool.map(verify_phase, range(len(self.follow))))
+
+        for n, b in enumerate(self.follow):
+            st = self.states[b]
+            K_t = len(o_draft[b])
+            LA0, LR0, o, ov = o_verify[n]
             rep.positions += K_t + 1
             _bump(rep.accept_hist, o["accept_len"])
             rep.n_rejections += o["rejected"]
             flagged_first = None      # first position whose decision is near its threshold
+            flagged_r6 = False        # ... and it was flagged for a distance within TOL of 0 or 1
             for i in range(K_t + 1):
                 c = f"b={b} i={i}"
                 self._close("H_t", float(rec["H_t"][b, i]), o["H_t"][i], ctx=c)
@@ -265,6 +292,7 @@ class Lockstep:
                 self._close("dist", float(rec["dist"][b, i]), o["dist"][i], ctx=c)
                 d = o["dist"][i]
                 near = (d < TOL) or (d > 1.0 - TOL)
+                near_end = near
                 if i <= o["accept_len"]:
                     # P(A|d) for the positions the oracle's loop reached
                     extra = [o["dist"][j] for j in range(i) if 0.0 < o["dist"][j] < 1.0]
@@ -275,6 +303,8 @@ class Lockstep:
                     sens = max(abs(Plo - P), abs(Phi - P))
                     self.report.err("p_acc_sensitivity", sens)
                     self._close("p_acc", float(rec["p_acc"][b, i]), P, tol=TOL + sens, ctx=c)
+                    rep.p_acc_checked += 1
+                    rep.p_acc_beyond_tol += abs(float(rec["p_acc"][b, i]) - P) > TOL
                     u = float(u_accept[b, i])
                     # the rejection rule in force: Bernoulli (u >= P) or the fixed threshold P < 1/2
                     cut = u if self.reject_rule == 0 else 0.5
@@ -286,6 +316,7 @@ class Lockstep:
                     rep.near_threshold += 1
                     if flagged_first is None:
                         flagged_first = i
+                        flagged_r6 = near_end
 
             # decisions
             agree = (int(al_h[b]) == o["accept_len"] and int(nt_h[b]) == o["next_token"]
@@ -301,12 +332,12 @@ class Lockstep:
                                f"sizes {(st.nE.value, st.nA.value, st.nR.value)}; p_acc gpu "
                                f"{rec['p_acc'][b, :K_t]} oracle {o['p_acc']} u {u_accept[b, :K_t]}")
                 rep.flips += 1
+                rep.r6_resyncs += flagged_r6
                 self._resync(b)
             else:
                 self._close("T_G", float(T_dev[b]), st.T_G.value, ctx=f"b={b}")
 
             if wl.vanilla:
-                ov = oracle.vanilla_round(hd[n][:K_t], ht[n], x_h[b, :K_t], u_vacc[b, :K_t], float(u_res[b]))
                 _bump(rep.vanilla_accept_hist, ov["accept_len"])
                 a_gpu = self.alpha[b].cpu().numpy()
                 near_v = None

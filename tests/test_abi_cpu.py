@@ -40,6 +40,34 @@ def test_strerror_and_null_arguments():
     assert lib.adasd_update_thresholds(None, None, None) == -1
 
 
+def test_error_codes_of_the_header_have_messages_and_match_the_binding():
+    text = open(os.path.join(ROOT, "include", "adasd.h")).read()
+    codes = dict((n, int(v)) for n, v in re.findall(r"#define (ADASD_ERR_[A-Z]+) \((-\d+)\)", text))
+    assert codes == {"ADASD_ERR_NULL": adasd.ERR_NULL, "ADASD_ERR_ALIGN": adasd.ERR_ALIGN,
+                     "ADASD_ERR_SHAPE": adasd.ERR_SHAPE, "ADASD_ERR_DTYPE": adasd.ERR_DTYPE,
+                     "ADASD_ERR_CAPACITY": adasd.ERR_CAPACITY, "ADASD_ERR_CUDA": adasd.ERR_CUDA,
+                     "ADASD_ERR_DEVICE": adasd.ERR_DEVICE}
+    msgs = {c: adasd.adasd_strerror(c) for c in codes.values()}
+    assert all(m != "unknown error" for m in msgs.values()) and len(set(msgs.values())) == len(msgs)
+    assert "device" in msgs[adasd.ERR_DEVICE] and "aligned" in msgs[adasd.ERR_ALIGN]
+    assert adasd.adasd_strerror(-6) == "unknown error" and adasd.adasd_strerror(-8) == "unknown error"
+
+
+def test_misaligned_pointers_are_refused_before_anything_runs():
+    """float / int32 arrays must sit on 4-byte boundaries, bf16 logits on 2-byte ones: the
+    context-free entry point checks that before it asks CUDA anything, so it shows here."""
+    ok = 0x10000                         # never dereferenced: every case below is refused on the host
+    def call(zd=ok, zt=ok, x=ok, dlen=None, ua=ok, ur=ok, al=ok, nt=ok, alpha=None, status=None,
+             dtype=adasd.ADASD_BF16):
+        return adasd.adasd_vanilla_verify_static(2, 1000, 4, dtype, zd, zt, 4000, 1000, 5000, 1000, x, dlen,
+                                                 ua, ur, al, nt, alpha, status, None)
+    assert call(zd=ok + 1) == adasd.ERR_ALIGN and call(zt=ok + 1) == adasd.ERR_ALIGN
+    assert call(zd=ok + 2, dtype=adasd.ADASD_FP32) == adasd.ERR_ALIGN      # fp32 logits: 4 bytes
+    for name in ("x", "dlen", "ua", "ur", "al", "nt", "alpha", "status"):
+        assert call(**{name: ok + 2}) == adasd.ERR_ALIGN, name
+    assert call(x=None) == adasd.ERR_NULL
+
+
 def test_create_validates_before_touching_cuda():
     for field, value, want in (("B", 0, -3), ("V", 0, -3), ("Kmax", 0, -3), ("Kmax", 33, -3),
                                ("list_capacity", 0, -3), ("dtype", 7, -4), ("kde_bandwidth", 2, -4),

@@ -66,11 +66,20 @@ def test_generator_host_and_device_rows_are_bit_identical(torch):
 # ------------------------------------------------------------------ workloads in lockstep
 
 def run_lockstep(wl, **kw):
+    import json
+    import os
+    import time
     from tests.lockstep import Lockstep
+    t0 = time.time()
     ls = Lockstep(wl, **kw)
     rep = ls.run()
     s = rep.summary()
     print(wl.name, s)
+    log = os.environ.get("ADASD_PARITY_LOG")       # one JSON line per workload, for the records
+    if log:
+        with open(log, "a") as f:
+            f.write(json.dumps(dict(workload=wl.name, B=wl.B, K=wl.K, V=wl.V, followed=len(ls.follow),
+                                    seconds=round(time.time() - t0, 1), **s)) + "\n")
     assert rep.flips <= max(2, rep.near_threshold), s
     return rep
 
@@ -116,27 +125,34 @@ def test_vanilla_mode_with_many_rows_takes_the_three_step_path(torch):
     assert len(rep.vanilla_accept_hist) >= 3
 
 
-def test_c2_single_stream_adaptive_window(torch):
-    wl = synth.WORKLOADS["C2"].scaled(rounds=40)
-    rep = run_lockstep(wl)
-    assert len(rep.window_hist) >= 2          # the stop check produced different windows
+# The four large workloads run EVERY round they state, in lockstep with the oracle: C2 and C3 on
+# all their sequences, C4 and C5 on eight sequences spread over the batch (the other sequences
+# run on the device all the same; the oracle follows the eight).
+
+def test_c2_single_stream_adaptive_window_all_512_rounds(torch):
+    wl = synth.WORKLOADS["C2"]
+    rep = run_lockstep(wl, check_lists_every=64)
+    assert rep.rounds == 512 and len(rep.window_hist) >= 2      # the stop check produced different windows
 
 
-def test_c3_batched_with_vanilla(torch):
-    wl = synth.WORKLOADS["C3"].scaled(rounds=24)
-    rep = run_lockstep(wl, follow=[0, 13, 31])
-    assert len(rep.accept_hist) >= 2 and len(rep.vanilla_accept_hist) >= 3
+def test_c3_batched_with_vanilla_all_256_rounds_all_32_sequences(torch):
+    wl = synth.WORKLOADS["C3"]
+    rep = run_lockstep(wl, check_lists_every=64)
+    assert rep.rounds == 256 and rep.positions == 256 * 32 * 9
+    assert len(rep.accept_hist) >= 5 and len(rep.vanilla_accept_hist) >= 5
 
 
-def test_c4_large_batch_large_vocab_sampled_sequences(torch):
-    wl = synth.WORKLOADS["C4"].scaled(rounds=5)
-    run_lockstep(wl, follow=[0, 77, 127])
+def test_c4_large_batch_large_vocab_all_128_rounds(torch):
+    wl = synth.WORKLOADS["C4"]
+    rep = run_lockstep(wl, follow=[0, 18, 37, 55, 73, 91, 110, 127], check_lists_every=32)
+    assert rep.rounds == 128 and rep.positions == 128 * 8 * 17
 
 
-def test_c5_streaming_adaptive_sampled_sequences(torch):
-    wl = synth.WORKLOADS["C5"].scaled(rounds=10)
-    rep = run_lockstep(wl, follow=[0, 100, 255])
-    assert max(rep.window_hist) <= 16
+def test_c5_streaming_adaptive_all_1024_rounds(torch):
+    # the lists end near 10^4 entries per sequence; the context's capacity covers 1024 * 16 appends
+    wl = synth.WORKLOADS["C5"]
+    rep = run_lockstep(wl, follow=[0, 36, 73, 109, 146, 182, 219, 255], check_lists_every=128)
+    assert rep.rounds == 1024 and max(rep.window_hist) <= 16 and len(rep.window_hist) >= 4
 
 
 def test_long_history_kde(torch):
@@ -284,6 +300,42 @@ def test_nan_and_all_minus_inf_rows_set_status_not_faults(torch, adasd, V, dt):
     assert np.isfinite(r["H_d"][0, 0]) and np.isfinite(r["H_t"][1, 1])
     assert c.ctx.status() & adasd.STATUS_NAN
     assert c.ctx.status() == 0                                   # reading clears it
+
+
+@pytest.mark.parametrize("V,dt", [(500, "float32"), (8200, "bfloat16")])
+def test_unusable_row_with_fused_update_leaves_thresholds_finite(torch, adasd, V, dt):
+    """A round whose first candidate has a NaN draft row (fused update on): the candidate is
+    rejected, nothing of it is recorded, T_G keeps its value; the clean round after it updates
+    the state exactly as the oracle does, and the draft-stop check still works."""
+    K = 3
+    rng = np.random.default_rng(31)
+    zd = rng.normal(size=(1, K, V)).astype(np.float32) * 2
+    zt = np.concatenate([zd + rng.normal(size=(1, K, V)).astype(np.float32),
+                         rng.normal(size=(1, 1, V)).astype(np.float32)], axis=1)
+    x = [[1, 2, 3]]
+    ut, ua = rng.random((1, K + 1)), np.full((1, K), 0.999)
+    st = oracle.SequenceState(capacity=64)
+    c = Case(torch, adasd, zd, zt, x, ut, ua, dtype=getattr(torch, dt))
+    o = c.oracle_round(0, st)                              # a clean round first: one rejection recorded
+    c.verify()
+    assert o["rejected"] and st.nE.value == 1
+    T0 = st.T_G.value
+    clean_d = c.zd.clone()
+    c.zd[0, 0, 100] = float("nan")
+    o = c.oracle_round(0, st)
+    r = c.verify()
+    assert c.ctx.status() & adasd.STATUS_NAN
+    assert np.isnan(r["H_d"][0, 0]) and int(c.al[0]) == 0 == o["accept_len"] and int(r["rejected"][0]) == 1
+    T, nE, nA, nR = (t.cpu().numpy() for t in c.ctx.get_thresholds())
+    assert (int(nE[0]), int(nA[0]), int(nR[0])) == (st.nE.value, st.nA.value, st.nR.value) == (1, 0, st.nR.value)
+    assert np.isfinite(T[0]) and abs(float(T[0]) - T0) < TOL and st.T_G.value == T0
+    c.zd.copy_(clean_d)                                    # a clean round again: the state moves on
+    o = c.oracle_round(0, st)
+    c.verify()
+    T, nE, nA, nR = (t.cpu().numpy() for t in c.ctx.get_thresholds())
+    assert (int(nE[0]), int(nA[0]), int(nR[0])) == (st.nE.value, st.nA.value, st.nR.value) and int(nE[0]) == 2
+    assert np.isfinite(T[0]) and abs(float(T[0]) - st.T_G.value) < TOL
+    assert c.ctx.status() == 0
 
 
 @pytest.mark.parametrize("V", [4096, 8200])      # generic kernel with the CTA-wide tail; streaming kernel with warp tails
@@ -644,3 +696,12 @@ def test_full_lists_set_the_capacity_flag_and_keep_running(torch, adasd):
     torch.cuda.synchronize()
     assert seen & adasd.STATUS_CAPACITY and not (seen & ~adasd.STATUS_CAPACITY)
     assert int(nR.max()) <= cap and int(nA.max()) <= cap and int(nR.max()) == cap
+    # L_E^R is capped the same way, and T_G stays the mean of what it holds: a checkpoint
+    # round trip leaves it where it was
+    assert int(nE.max()) == cap
+    for b in range(B):
+        before = ctx.state_export(b)
+        ctx.state_import(b, before["T_G"], before["LE"], before["LA"], before["LR"])
+        after = ctx.state_export(b)
+        assert abs(after["T_G"] - before["T_G"]) < 1e-6 and len(after["LE"]) == len(before["LE"])
+        assert abs(before["T_G"] - float(np.mean(before["LE"]))) < 1e-5

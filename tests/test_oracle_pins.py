@@ -414,6 +414,30 @@ def test_boundary_distances_skip_kde_lists_but_entropy_is_recorded():
     assert (st.nE.value, st.nA.value, st.nR.value) == (2, 0, 0)
 
 
+def test_unusable_rows_are_rejected_and_leave_the_state_alone():
+    """A draft row with NaN (or a target row without a finite logit) has no entropy and no
+    distance: the candidate is rejected on a token mismatch, nothing is appended and T_G
+    keeps its value (a NaN in L_E^R would switch the stop check off for good)."""
+    V = 8
+    r = np.random.default_rng(5)
+    st = oracle.SequenceState(capacity=64)
+    zd = r.normal(size=(2, V)).astype(np.float32)
+    zt = r.normal(size=(3, V)).astype(np.float32)
+    out = oracle.verify_round(st, zd, zt, [V + 5, V + 5], [0.5, 0.5, 0.5], [0.9, 0.9])   # ordinary rejection first
+    assert out["rejected"] and st.nE.value == 1
+    T0, sizes = st.T_G.value, (st.nE.value, st.nA.value, st.nR.value)
+    zd[0, 3] = np.nan
+    out = oracle.verify_round(st, zd, zt, [V + 5, V + 5], [0.5, 0.5, 0.5], [0.9, 0.9])
+    assert out["rejected"] and out["accept_len"] == 0 and math.isnan(out["H_d"][0]) and math.isnan(out["dist"][0])
+    assert (st.nE.value, st.nA.value, st.nR.value) == sizes and st.T_G.value == T0
+    zd[0, 3] = 0.0
+    zt[0, :] = -np.inf
+    out = oracle.verify_round(st, zd, zt, [V + 5, V + 5], [0.5, 0.5, 0.5], [0.9, 0.9])
+    assert out["rejected"] and out["y"][0] == -1 and math.isnan(out["dist"][0])
+    assert math.isfinite(out["H_d"][0])                      # the draft row itself is fine ...
+    assert (st.nE.value, st.nA.value, st.nR.value) == sizes and st.T_G.value == T0   # ... but the position has no distance
+
+
 def test_match_always_accepts_and_update_flag():
     V, K = 16, 4
     r = np.random.default_rng(11)

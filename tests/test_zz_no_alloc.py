@@ -5,8 +5,9 @@ that gave the whole GPU to its own pool, a plugin that must leave the allocator 
 They cannot create a context, so the library offers one context-free call whose scratch
 is a fixed array inside the library image.  This file checks, through the C ABI, that
 the call returns what adasd_vanilla_verify returns on the same inputs, twice in a row
-(the second call meets the first call's leftovers in the shared array), and that sizes
-beyond the stated maximum are refused.
+(the second call meets the first call's leftovers in the shared array), that both agree
+with the float64 oracle's vanilla round on every sequence, and that sizes beyond the
+stated maximum are refused.
 
 Collected last on purpose: a run that stops at the first failure has then already run
 every other test.  The test builds its own inputs and passes on its own in a fresh
@@ -15,6 +16,7 @@ process as well as after the rest of the suite.
 import numpy as np
 import pytest
 
+import oracle
 import paper_2512_11280_b200 as adasd
 import synth
 
@@ -40,7 +42,16 @@ def _inputs(wl, round_, dev):
     return zd, zt, x, dlen, U
 
 
-@pytest.mark.parametrize("dtype,V", [(synth.FP32, 32000), (synth.BF16, 5000), (synth.BF16, 4099)])
+def _raw(t):
+    """Device logits -> the oracle's raw input (bf16 bits or float32)."""
+    import torch
+    return t.view(torch.int16).cpu().numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.cpu().numpy()
+
+
+# fp32 rows; bf16 rows that are not 16-byte aligned (scalar loads); bf16 rows of a multiple of 8
+# logits (16-byte vector loads)
+@pytest.mark.parametrize("dtype,V", [(synth.FP32, 32000), (synth.BF16, 5000), (synth.BF16, 4099),
+                                     (synth.BF16, 4096)])
 def test_static_entry_matches_context_entry_twice(dtype, V):
     import torch
     dev = torch.device("cuda", 0)
@@ -74,6 +85,18 @@ def test_static_entry_matches_context_entry_twice(dtype, V):
         err = (alpha - ref_alpha).abs()[live]
         assert err.numel() == int(dlen.sum()) and not torch.isnan(err).any()
         assert float(err.max()) <= TOL if err.numel() else True
+        # the oracle's vanilla round of every sequence (Sec. 2.1.3), not just the other entry point
+        x_h, dl_h, al_h, nt_h, a_h = (t.cpu().numpy() for t in (x, dlen, al, nt, alpha))
+        ua_h, ur_h = U["vanilla_accept"].cpu().numpy(), U["resample"].cpu().numpy()
+        for b in range(B):
+            K_t = int(dl_h[b])
+            o = oracle.vanilla_round(_raw(zd[b, :K_t]), _raw(zt[b]), x_h[b, :K_t], ua_h[b, :K_t], float(ur_h[b]))
+            n_seen = min(o["accept_len"] + 1, K_t)
+            assert np.allclose(a_h[b, :n_seen], o["alpha"][:n_seen], atol=TOL), (b, a_h[b], o["alpha"])
+            near = any(abs(float(ua_h[b, i]) - o["alpha"][i]) < TOL for i in range(n_seen))
+            assert int(al_h[b]) == o["accept_len"] or near, (b, al_h[b], o)
+            if int(al_h[b]) == o["accept_len"] and o["margin"] > 2e-6:
+                assert int(nt_h[b]) == o["next_token"], (b, nt_h[b], o)
     assert ctx.status() == 0
     ctx.close()
 
