@@ -80,7 +80,9 @@ def run_lockstep(wl, **kw):
         with open(log, "a") as f:
             f.write(json.dumps(dict(workload=wl.name, B=wl.B, K=wl.K, V=wl.V, followed=len(ls.follow),
                                     seconds=round(time.time() - t0, 1), **s)) + "\n")
-    assert rep.flips <= max(2, rep.near_threshold), s
+    # every disagreement was checked where it arose (it sat on a flagged decision or followed a
+    # sample whose uniform lay on a CDF edge); there cannot be more of them than of those
+    assert rep.flips <= rep.near_threshold + rep.tie_flips, s
     return rep
 
 
