@@ -249,9 +249,11 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
         van_accept = p.u_accept[(size_t)b * Kmax + i] < alpha;
     }
 
-    // pass C: sum p a', sum q b', sum s (1 - log2 s), sum p q   [a' = log2 p, b' = log2 q, s = p + q]
-    // JSD = (ln2 / 2) * (sum p a' + sum q b' + sum s (1 - log2 s)),  H = -ln2 * sum p a';
-    // sum p q == 0 means disjoint supports, where JSD is ln 2 exactly.
+    // pass C: sum p a', sum q b' (entropies: a' = log2 p, b' = log2 q), sum p q (== 0 means disjoint
+    // supports, where D_JS is ln 2 exactly) and the divergence itself from non-negative terms,
+    //   D_JS = 1/4 sum s phi(u),  s = p + q,  u = (q - p) / s,  phi(u) = (1-u) ln(1-u) + (1+u) ln(1+u):
+    // for |u| < 1/2 the series u^2 + u^4/6 + u^6/15 + u^8/28 + u^10/45, else the two logarithms.
+    // Nothing cancels however close the rows are (Sec. 2.2, first printed form, term by term).
     // vanilla on a rejected row: residual mass max(0, p - q), per warp and in total.
     float vC[4] = {0.f, 0.f, 0.f, 0.f};
     const bool need_resid = (MODE == MODE_VANILLA) && !bonus && !van_accept;
@@ -270,8 +272,22 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
                     float qq = ex2(bq);
                     if (MODE == MODE_ADASD) {
                         vC[1] = fmaf(qq, bq, vC[1]);
-                        float s = pp + qq;
-                        vC[2] = fmaf(s, 1.f - lg2(fmaxf(s, kTiny)), vC[2]);
+                        const float s = pp + qq;
+                        if (s > 0.f) {
+                            const float rs = __fdividef(1.f, s), uu = (qq - pp) * rs, w = uu * uu;
+                            float ph;
+                            if (w < 0.25f) {
+                                ph = fmaf(w, 1.f / 45.f, 1.f / 28.f);
+                                ph = fmaf(ph, w, 1.f / 15.f);
+                                ph = fmaf(ph, w, 1.f / 6.f);
+                                ph = fmaf(ph, w, 1.f);
+                                ph *= w;
+                            } else {
+                                const float lo = 2.f * pp * rs, hi = 2.f * qq * rs;     // 1 - u and 1 + u, each to full relative accuracy
+                                ph = kLn2 * ((lo > 0.f ? lo * lg2(lo) : 0.f) + (hi > 0.f ? hi * lg2(hi) : 0.f));
+                            }
+                            vC[2] = fmaf(s, ph, vC[2]);
+                        }
                         vC[3] = fmaf(pp, qq, vC[3]);
                     } else {
                         vC[3] += fmaxf(pp - qq, 0.f);
@@ -348,7 +364,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
             if (p.user.lse_t) p.user.lse_t[it] = lse_t;
             if (!bonus) {
                 float Hd = -kLn2 * vC[1], lse_d = fmaf(kLn2, lSd, md);
-                float jsd = 0.5f * kLn2 * (vC[0] + vC[1] + vC[2]);
+                float jsd = 0.25f * vC[2];
                 jsd = differ ? fminf(fmaxf(jsd, 0.f), kLn2) : 0.f;   // identical rows: exactly 0
                 if (!(vC[3] > 0.f)) jsd = kLn2;                      // disjoint supports: exactly ln 2
                 float dist = sqrtf(jsd / kLn2);

@@ -6,14 +6,21 @@
 // split the CTA's slice into contiguous runs of "iterations" (one iteration = 32 lanes x 16
 // bytes of each row).  Every logit row is read from HBM exactly once, by 1-D bulk copies
 // (cp.async.bulk) into per-warp buffers that hold two whole positions; the copy of position
-// n + 2 is issued the moment position n is done with, so HBM never waits for the arithmetic.
-// Values live in the log2 domain: t = z log2 e - M, 2^t kept in registers for the first
-// iterations and, for the rest, parked in the buffer over logits that have been used up.
+// n + 2 is issued the moment the logits of position n have been turned into 2^t values, so
+// HBM never waits for the arithmetic.  Values live in the log2 domain: t = z log2 e - M.  The
+// 2^t values of a position wait for the row totals in TENSOR MEMORY (the SM's 256 KB that the
+// tensor cores would use as accumulators; nothing here is a contraction, so it is free): the
+// first iterations of a warp's share go there (tcgen05.st), the rest stay in registers.
+// That leaves room for the head of position n + 1 to be worked through while the totals of
+// position n are exchanged: the special-function pipe does not idle during the exchange.
 //
 //  * 12 COMPUTE warps per CTA (three per scheduler) do nothing but the passes over their share of a position
-//    (A: maxima and flags; B: 2^t, S = sum 2^t and T = sum 2^t t; C: (p+q) log2 (p+q) in
-//    AdaSD mode, the residual mass max(0, p - q) of a rejected row in vanilla mode), the
-//    refill of their own buffers and, for the one warp that holds it, the inverse-CDF crossing.
+//    (A: maxima and flags; B: 2^t, S = sum 2^t, T = sum 2^t t and the largest |z_t - z_d|;
+//    C: (p+q) log2 (p+q) in AdaSD mode - or, when the two rows are nearly equal everywhere, the
+//    well-conditioned sum of (p+q) phi((q-p)/(q+p)) - and the residual mass max(0, p - q) of a
+//    rejected row in vanilla mode), the refill of their own buffers and, for the one warp that
+//    holds it, the inverse-CDF crossing.  Per position: A(n+1), head of B(n+1) | wait for the
+//    scale factors of n | C(n) | tail of B(n+1), publish its partials, refill.
 //  * 1 CONTROL warp per CTA finds the cluster's positions, folds the warp partials into the
 //    CTA's totals, exchanges them with the other CTAs of the cluster (st.async into their
 //    shared memory, counted on their mbarriers: no cluster-wide barrier in the loop) and
@@ -24,10 +31,12 @@
 //    T_G; vanilla: longest accepted prefix) of completed sequences, off everybody's critical
 //    path; AdaSD tails are handed to the idle tail warps of the cluster's other CTAs.
 //
-// The CTA has 16 warps = four warpgroups.  All threads start with 128 registers; the warpgroup
-// of service warps (control, tail and two idle warps) hands registers back with setmaxnreg and
-// the three warpgroups of compute warps take them: 144 registers per compute thread, 80 per
-// service thread.
+// The CTA has 16 warps of 128 registers per thread: the whole register file.
+//
+// Tensor memory: 512 columns x 128 lanes of 32 bits, allocated once per CTA by the control warp.
+// A warp may only touch the 32 lanes of its quarter (warp index mod 4), so the three compute
+// warps of a quarter split the columns: 160 each = two halves (position parity) of kSHead
+// slots of 16 columns; a slot holds one iteration's 8 target and 8 draft values per lane.
 //
 // Every wait (buffer filled, partials in, totals in, message ready, sums in, queue) is bounded:
 // a warp whose wait expires sets ADASD_STATUS_TIMEOUT, stops waiting and copying, and walks
@@ -42,12 +51,16 @@ constexpr int kSW = 12;                          // compute warps per CTA
 constexpr int kSCtl = kSW;                       // warp index of the control warp
 constexpr int kSTail = kSW + 1;                  // warp index of the tail warp
 constexpr int kSThreads = (kSW + 4) * 32;        // 512: three warpgroups of compute warps, one of service warps
-constexpr int kSRegIter = 5;                     // iterations whose 2^t values stay in registers
-constexpr int kSMaxIter = 10;                    // largest number of iterations per warp and row
-// Iteration k >= kSRegIter parks its 2^t values in the buffer pieces of iterations 2 (k - kSRegIter)
-// and 2 (k - kSRegIter) + 1, which must have been consumed before it: 2 (k - kSRegIter) + 1 < k.
-static_assert(2 * (kSMaxIter - 1 - kSRegIter) + 1 <= kSMaxIter - 1, "parked 2^t values would overwrite unread logits");
+constexpr int kSHead = 5;                        // iterations whose 2^t values wait in tensor memory
+constexpr int kSRegIter = 5;                     // ... and in registers, at most
+constexpr int kSMaxIter = kSHead + kSRegIter;    // largest number of iterations per warp and row
+constexpr int kSTmemCols = 512;                  // columns allocated (all of them: one CTA per SM)
+constexpr int kSTmemHalf = kSHead * 16;          // columns of one position's head: 16 per iteration
+constexpr int kSTmemWarp = 2 * kSTmemHalf;       // columns of one compute warp: two positions in flight
+static_assert((kSW / 4) * kSTmemWarp <= kSTmemCols, "the compute warps of a lane quarter share its columns");
+static_assert(kSW % 4 == 0, "compute warps are spread evenly over the four lane quarters");
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
+constexpr float kSNearDz = 0.5f;                 // rows count as nearly equal when no logit differs by more
 constexpr int kSPosRing = 16;                    // positions the control warp keeps described
 constexpr int kSWorkQ = 16;                      // tail work queue entries per CTA
 constexpr int kSFinRing = 4;                     // positions whose sums may await finalisation
@@ -67,7 +80,8 @@ struct __align__(16) PosCtx {
 // holds the inverse-CDF crossing (sel), the weight before its share and the target.
 struct __align__(16) WarpMsg {
     float at, ad, ft;             // first part: ready when scal_bar completes
-    int32_t act;                  // vanilla: 0 nothing left to do, 1 sample from p, 2 residual pass
+    int32_t act;                  // vanilla: 0 nothing left to do, 1 sample from p, 2 residual pass;
+                                  // AdaSD: 1, plus 4 when the rows are nearly equal (pass C in its u form)
     float target;                 // second part: ready when sel_bar completes
     int32_t sel;
     float base;
@@ -81,6 +95,8 @@ struct __align__(16) SpecShared {
     WarpMsg wmsg[2][kCW];
     float4 tabC[kSFinRing][kCTab];    // leader: per-warp (sum s log2 s, sum 2^t_p 2^t_q, token or -1), by position
     float fin[kSFinRing][12];         // leader: row totals (and alpha, accept flag) kept for finalisation
+    RowPart finc[kSFinRing][kCMaxCluster];   // leader: every CTA's totals, kept for the float64 finalisation
+    uint32_t tmem_base;               // tensor-memory address the allocation returned
     float rw[kCW];                    // vanilla: residual mass of each compute warp's share
     float4 rtab[kCMaxCluster];        // vanilla: every CTA's residual mass (written over DSMEM)
     unsigned long long entry_bar[2];  // one arrival per compute warp: wtab[par] complete
@@ -126,6 +142,115 @@ __device__ __forceinline__ uint32_t ld_cluster_u32(uint32_t remote_addr) {
     return v;
 }
 __device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+
+// ---- tensor memory as a scratchpad ---------------------------------------------------------
+// Allocation and release are warp-wide; the address lands in shared memory.
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// 16 consecutive columns of this thread's lane: a[0..7] then b[0..7]
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&a)[8], const float (&b)[8]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "f"(a[0]), "f"(a[1]), "f"(a[2]), "f"(a[3]), "f"(a[4]), "f"(a[5]), "f"(a[6]), "f"(a[7]),
+          "f"(b[0]), "f"(b[1]), "f"(b[2]), "f"(b[3]), "f"(b[4]), "f"(b[5]), "f"(b[6]), "f"(b[7])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const float (&a)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "f"(a[0]), "f"(a[1]), "f"(a[2]), "f"(a[3]), "f"(a[4]), "f"(a[5]), "f"(a[6]), "f"(a[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// The loads are asynchronous: the registers hold the values only after tmem_wait_ld, which
+// takes them as operands so that nothing that uses them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&a)[8], float (&b)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=f"(a[0]), "=f"(a[1]), "=f"(a[2]), "=f"(a[3]), "=f"(a[4]), "=f"(a[5]), "=f"(a[6]), "=f"(a[7]),
+          "=f"(b[0]), "=f"(b[1]), "=f"(b[2]), "=f"(b[3]), "=f"(b[4]), "=f"(b[5]), "=f"(b[6]), "=f"(b[7])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&a)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(a[0]), "=f"(a[1]), "=f"(a[2]), "=f"(a[3]), "=f"(a[4]), "=f"(a[5]), "=f"(a[6]), "=f"(a[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld(float (&a)[8], float (&b)[8]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7]),
+                   "+f"(b[0]), "+f"(b[1]), "+f"(b[2]), "+f"(b[3]), "+f"(b[4]), "+f"(b[5]), "+f"(b[6]), "+f"(b[7])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld(float (&a)[8]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+f"(a[0]), "+f"(a[1]), "+f"(a[2]), "+f"(a[3]), "+f"(a[4]), "+f"(a[5]), "+f"(a[6]), "+f"(a[7])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// The published scalars of one position from the CTAs' statistics (lane c holds CTA c) and the
+// warps' pass-C sums, worked out in float64 by the whole tail warp.  In fp32 the totals
+// (entropies of up to 17 bits, log2 of sums of up to 2^17) carry errors of about 1e-6 each, which
+// the difference H(m) - (H(p) + H(q)) / 2 keeps.
+struct FinOut {
+    float Ht, lse_t, Hd, lse_d, jsd, dist;
+};
+__device__ __forceinline__ FinOut finalize_math(const RowPart* finc, int CS, float Mt, float Md, double A, float PQ,
+                                             uint32_t fl, bool near) {
+    const int lane = threadIdx.x & 31;
+    // row totals: S = sum f_c S_c, T = sum f_c (T_c + (M_c - M) S_c) with f_c = 2^(M_c - M)
+    double St = 0.0, Tt = 0.0, Sd = 0.0, Td = 0.0;
+    if (lane < CS) {
+        const float4* fc = reinterpret_cast<const float4*>(finc + lane);
+        const float4 e0 = fc[0], e1 = fc[1];
+        const double dt = (double)e0.x - (double)Mt, dd = (double)e0.w - (double)Md;
+        const double ft = e0.x > kFloorL ? exp2(dt) : 0.0, fd = e0.w > kFloorL ? exp2(dd) : 0.0;
+        St = ft * (double)e0.y;
+        Tt = ft * ((double)e0.z + dt * (double)e0.y);
+        Sd = fd * (double)e1.x;
+        Td = fd * ((double)e1.y + dd * (double)e1.x);
+    }
+    St = warp_sum_f64(St);
+    Tt = warp_sum_f64(Tt);
+    Sd = warp_sum_f64(Sd);
+    Td = warp_sum_f64(Td);
+    const double kLn2d = 0.69314718055994530942;
+    const double lSt = log2(St), lSd = log2(Sd);
+    const double Hbt = lSt - Tt / St, Hbd = lSd - Td / Sd;      // entropies in bits
+    FinOut o;
+    o.Ht = (float)(kLn2d * Hbt);
+    o.lse_t = (float)(kLn2d * ((double)Mt + lSt));
+    o.Hd = (float)(kLn2d * Hbd);
+    o.lse_d = (float)(kLn2d * ((double)Md + lSd));
+    // nearly equal rows: A is sum s phi(u), D_JS = A / 4 (nats), nothing cancels; else
+    // D_JS = H(m) - (H(p) + H(q)) / 2 with H(m) = (ln 2 / 2) (2 - sum s log2 s), s = p + q
+    const double jd = near ? 0.25 * A : 0.5 * kLn2d * ((2.0 - A) - (Hbt + Hbd));
+    float jsd = (float)fmin(fmax(jd, 0.0), kLn2d);
+    if (!(fl & 2u)) jsd = 0.f;                              // identical rows: exactly 0
+    if (!(PQ > 0.f)) jsd = kLn2;                            // disjoint supports: ln 2
+    o.jsd = jsd;
+    o.dist = jsd >= kLn2 ? 1.f : fminf((float)sqrt((double)jsd / kLn2d), 1.f);
+    return o;
+}
 
 // The per-sequence tail of a round, run by ONE warp: lane i owns candidate i.  Same
 // arithmetic as verify_tail (KDE sums over L_D^A and L_D^R, Bayes posterior with the
@@ -253,7 +378,9 @@ __device__ __forceinline__ void verify_tail_warp(const TailConfig& cfg, const Ta
 template <int ITER, int MODE>
 __global__ void __launch_bounds__(kSThreads, 1)
 spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
-    constexpr int KR = ITER < kSRegIter ? ITER : kSRegIter;   // iterations kept in registers
+    constexpr int KH = ITER < kSHead ? ITER : kSHead;          // head iterations: 2^t values in tensor memory
+    constexpr int KR = ITER - KH;                              // tail iterations: 2^t values in registers
+    static_assert(KR <= kSRegIter, "too many iterations for the register file");
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ SpecShared sh;
 
@@ -351,16 +478,22 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             set_pos(n, r);
         }
         lastp = r;
+        // all of the SM's tensor memory (this kernel runs one CTA per SM): the address comes back
+        // in shared memory and is read by everybody after the barrier below
+        tmem_alloc(&sh.tmem_base, (uint32_t)kSTmemCols);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    cluster.sync();   // barriers and positions are set up in every CTA of the cluster
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    cluster.sync();   // barriers, positions and tensor memory are set up in every CTA of the cluster
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_base);
 
-    // 512 threads start with 128 registers each.  The warpgroup of service warps (two of its four
-    // warps have work) gives registers back, the three warpgroups of compute warps take them:
-    // 12 x 32 x 144 + 4 x 32 x 80 = 65536.
+    // 512 threads x 128 registers fill the register file: every warp keeps what it started with
+    // (the compute warps' kept 2^t values take at most 80 registers now that the head of a position
+    // waits in tensor memory; the tail warp's float64 finalisation needs about as many).
+
     if (warp < kSW) asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
     else asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
-
     bool alive = true;         // false after a wait expired: this warp stops waiting and copying
     auto expired = [&]() {
         alive = false;
@@ -392,15 +525,21 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         const size_t woff = (size_t)wi0 * 512;                     // its byte offset in the CTA's slice
 
         // Two buffers per warp, one position each: [target share | draft share], ITER * 512 bytes
-        // per row.  Position n lives in buffer n & 1 and is replaced by position n + 2 as soon as
-        // pass C of position n is done, one whole position before it is needed.
+        // per row.  Position n lives in buffer n & 1; once pass B has turned its logits into 2^t
+        // values the buffer is refilled with position n + 2, one whole position before that is
+        // needed.
         const int kRowB = I_w * 512;              // bytes of one row in this warp's buffers
         unsigned char* const bufs = dyn_smem + (size_t)wi0 * 2048;
         auto buf_of = [&](int n) -> unsigned char* { return bufs + (size_t)(n & 1) * (2 * kRowB) + (size_t)lane * 16; };
         auto bar_of = [&](int n) -> uint64_t* { return reinterpret_cast<uint64_t*>(&sh.bar[warp][n & 1]); };
         auto pcx = [&](int n) -> const PosCtx& { return sh.pc[n & (kSPosRing - 1)]; };
+        // This warp's tensor-memory columns: the lanes of its quarter, 160 columns of its own.
+        // Head iteration k of position n sits in slot k of half n & 1.
+        const uint32_t tm_warp = tmem0 + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((warp >> 2) * kSTmemWarp);
+        auto tm_of = [&](int n, int k) -> uint32_t { return tm_warp + (uint32_t)((n & 1) * kSTmemHalf + k * 16); };
 
         // lanes 0 and 1 fetch the two rows of position n (lane 1 idles for a bonus row)
+        int n_issued = 0, n_landed = 0;           // positions asked for / seen to have landed (for the give-up path)
         auto issue_pos = [&](int n) {
             const PosCtx& c = pcx(n);
             if (!alive || nwu == 0 || c.pos >= total) return;
@@ -413,6 +552,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             if (lane < (bonus ? 1 : 2))
                 bulk_g2s(dst + lane * kRowB,
                          reinterpret_cast<const unsigned char*>(lane ? c.src_d : c.src_t) + woff, row_bytes, bar);
+            n_issued = n + 1;
         };
         issue_pos(0);
         issue_pos(1);
@@ -427,157 +567,164 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         };
 
         // ---- pass A: packed maxima and flags of one position ---------------------------------
-        uint32_t a_mT = 0xFF80FF80u, a_mD = 0xFF80FF80u, a_df = 0u;   // -inf pairs
-        bool a_done = false;
-        // with blocking == false it gives up at once if the position has not landed yet
-        auto pass_a = [&](auto bonus_c, int n, bool blocking) {
-            constexpr bool BONUS = decltype(bonus_c)::value;
-            if (!alive || a_done) return;
-            if (nwu > 0) {
-                const uint32_t par = (uint32_t)(n >> 1) & 1u;
-                bool ok = blocking ? mbar_wait_bounded(bar_of(n), par) : (mbar_test_wait(bar_of(n), par) != 0);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) {
-                    if (blocking) expired();     // the copy never landed
-                    return;
-                }
-            }
-            a_done = true;
-            const unsigned char* sb = buf_of(n);
-#pragma unroll
-            for (int k = 0; k < ITER; ++k) {
-                if (k_on(k)) {
-                    uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
-                    mask_unit(k, T);
-                    a_mT = bmax2(bmax2(a_mT, T.x), bmax2(T.y, bmax2(T.z, T.w)));
-                    if (!BONUS) {
-                        uint4 D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
-                        mask_unit(k, D);
-                        a_mD = bmax2(bmax2(a_mD, D.x), bmax2(D.y, bmax2(D.z, D.w)));
-                        a_df |= (T.x ^ D.x) | (T.y ^ D.y) | (T.z ^ D.z) | (T.w ^ D.w);
-                    }
-                }
-            }
-        };
-        auto pass_a_any = [&](bool bonus, int n, bool blocking) {
-            if (bonus) pass_a(std::true_type{}, n, blocking);
-            else pass_a(std::false_type{}, n, blocking);
-        };
-
-        // The warp's shifts and flags from the packed accumulators.  Every kept value is
+        // The warp's shifts and flags from the packed maxima.  Every kept value is
         // 2^((z - max) log2 e) with the share's own largest logit, exactly 1 for that logit;
         // shares combine in the log2 domain through the differences of M = fl(max * log2 e).
         // A slice without a finite logit gets M = kFloorL and all-zero values.
         float nmt_w = 0.f, nmd_w = 0.f;           // addends of pass B (-max, or 0 for an empty slice)
         uint32_t flags_w = 0;
-        auto finish_a = [&](bool bonus) {
+        auto pass_a = [&](auto bonus_c, int n) {
+            constexpr bool BONUS = decltype(bonus_c)::value;
+            uint32_t a_mT = 0xFF80FF80u, a_mD = 0xFF80FF80u, a_df = 0u;   // -inf pairs
+            if (alive && nwu > 0) {
+                bool ok = mbar_wait_bounded(bar_of(n), (uint32_t)(n >> 1) & 1u);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) expired();                // the copy never landed
+                else n_landed = n + 1;
+            }
+            if (alive) {
+                const unsigned char* sb = buf_of(n);
+#pragma unroll
+                for (int k = 0; k < ITER; ++k) {
+                    if (k_on(k)) {
+                        uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
+                        mask_unit(k, T);
+                        a_mT = bmax2(bmax2(a_mT, T.x), bmax2(T.y, bmax2(T.z, T.w)));
+                        if (!BONUS) {
+                            uint4 D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
+                            mask_unit(k, D);
+                            a_mD = bmax2(bmax2(a_mD, D.x), bmax2(D.y, bmax2(D.z, D.w)));
+                            a_df |= (T.x ^ D.x) | (T.y ^ D.y) | (T.z ^ D.z) | (T.w ^ D.w);
+                        }
+                    }
+                }
+            }
             const float2 a = unpack2(a_mT), d = unpack2(a_mD);
             uint32_t bad = (a.x != a.x || a.y != a.y || d.x != d.x || d.y != d.y) ? 1u : 0u;
             const float vt = warp_max_f32(fmaxf(a.x, a.y));
-            const float vd = bonus ? vt : warp_max_f32(fmaxf(d.x, d.y));
+            const float vd = BONUS ? vt : warp_max_f32(fmaxf(d.x, d.y));
             if (vt == INFINITY || vd == INFINITY || !alive) bad = 1u;
             const bool has_t = vt > ADASD_FLOOR_BF, has_d = vd > ADASD_FLOOR_BF;
             nmt_w = has_t ? -vt : 0.f;
             nmd_w = has_d ? -vd : 0.f;
             // bits 4 and 8 (not published): the target / draft share has no finite logit
             flags_w = __reduce_or_sync(0xFFFFFFFFu, bad | (a_df ? 2u : 0u)) | (has_t ? 0u : 4u) | (has_d ? 0u : 8u);
-            a_mT = a_mD = 0xFF80FF80u;
-            a_df = 0u;
-            a_done = false;
         };
 
-        // 2^t values of one unit: 8 logits (four packed words) relative to the shift in `nm`
-        // nv = -(largest logit of the share): t = (z - max) log2 e is exactly 0 for the largest
-        // logit, so that a one-hot row gets S = 1, T = 0, p = 1 and H = 0 exactly.
-        auto exps = [&](const uint4& W, const float2 nv, float (&e)[8], float2& S, float2& Tq) {
-            const float2 L2 = make_float2(kLog2e, kLog2e);
-            const uint32_t w[4] = {W.x, W.y, W.z, W.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float2 z = unpack2(bclamp2(w[j]));
-                const float2 t = __fmul2_rn(__fadd2_rn(z, nv), L2);
-                const float2 v = make_float2(ex2(t.x), ex2(t.y));
-                e[2 * j] = v.x;
-                e[2 * j + 1] = v.y;
-                S = __fadd2_rn(S, v);
-                Tq = __ffma2_rn(v, t, Tq);
-            }
-        };
-
-        // ---- pass B: the warp's S and T; the 2^t values of the first KR iterations are kept ----
-        float et[KR][8], ed[KR][8];
-        float sB[4];                       // after pass_b: warp totals St, Tt, Sd, Td
-        auto pass_b = [&](auto bonus_c, int n) {
+        // ---- pass B: 2^t of every logit of the share, S = sum 2^t, T = sum 2^t t, max |z_t - z_d| --
+        // Head iterations [0, KH) park their values in tensor memory, tail iterations [KH, ITER)
+        // keep them in registers.  t = (z - max) log2 e is exactly 0 for the largest logit of the
+        // share, so that a one-hot row gets S = 1, T = 0, p = 1 and H = 0 exactly.
+        float et[KR > 0 ? KR : 1][8], ed[KR > 0 ? KR : 1][8];
+        float2 bSt = make_float2(0.f, 0.f), bTt = bSt, bSd = bSt, bTd = bSt;   // lane partials of the position in pass B
+        float bdz = 0.f;
+        auto pass_b = [&](auto bonus_c, auto k0_c, auto k1_c, int n) {
             constexpr bool BONUS = decltype(bonus_c)::value;
-            float2 St = make_float2(0.f, 0.f), Tt = St, Sd = St, Td = St;
+            constexpr int K0 = decltype(k0_c)::value, K1 = decltype(k1_c)::value;
+            if (K0 == 0) {
+                bSt = bTt = bSd = bTd = make_float2(0.f, 0.f);
+                bdz = 0.f;
+            }
             const float2 nmt = make_float2(nmt_w, nmt_w), nmd = make_float2(nmd_w, nmd_w);
+            const float2 L2 = make_float2(kLog2e, kLog2e), neg1 = make_float2(-1.f, -1.f);
             const unsigned char* sb = buf_of(n);
 #pragma unroll
-            for (int k = 0; k < ITER; ++k) {
+            for (int k = K0; k < K1; ++k) {
                 if (k_on(k)) {
                     float e1[8], e2[8];
                     uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
                     mask_unit(k, T);
-                    exps(T, nmt, e1, St, Tt);
+                    uint4 D = make_uint4(0u, 0u, 0u, 0u);
                     if (!BONUS) {
-                        uint4 D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
+                        D = *reinterpret_cast<const uint4*>(sb + kRowB + k * 512);
                         mask_unit(k, D);
-                        exps(D, nmd, e2, Sd, Td);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) e2[j] = 0.f;
                     }
-                    if (k < KR) {
+                    const uint32_t tw[4] = {T.x, T.y, T.z, T.w}, dw[4] = {D.x, D.y, D.z, D.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 zt = unpack2(bclamp2(tw[j]));
+                        const float2 tt = __fmul2_rn(__fadd2_rn(zt, nmt), L2);
+                        const float2 vt = make_float2(ex2(tt.x), ex2(tt.y));
+                        e1[2 * j] = vt.x;
+                        e1[2 * j + 1] = vt.y;
+                        bSt = __fadd2_rn(bSt, vt);
+                        bTt = __ffma2_rn(vt, tt, bTt);
+                        if (!BONUS) {
+                            const float2 zd = unpack2(bclamp2(dw[j]));
+                            const float2 td = __fmul2_rn(__fadd2_rn(zd, nmd), L2);
+                            const float2 vd = make_float2(ex2(td.x), ex2(td.y));
+                            e2[2 * j] = vd.x;
+                            e2[2 * j + 1] = vd.y;
+                            bSd = __fadd2_rn(bSd, vd);
+                            bTd = __ffma2_rn(vd, td, bTd);
+                            const float2 df = __ffma2_rn(zd, neg1, zt);        // exact: both are bf16 values
+                            bdz = fmaxf(bdz, fmaxf(fabsf(df.x), fabsf(df.y)));
+                        } else {
+                            e2[2 * j] = 0.f;
+                            e2[2 * j + 1] = 0.f;
+                        }
+                    }
+                    if (k < KH) {
+                        if (BONUS) tmem_st8(tm_of(n, k), e1);
+                        else tmem_st16(tm_of(n, k), e1, e2);
+                    } else {
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
-                            et[k < KR ? k : 0][j] = e1[j];
-                            ed[k < KR ? k : 0][j] = e2[j];
-                        }
-                    } else {
-                        // no register left: the values go over logits this lane has already turned
-                        // into 2^t values (two 512-byte pieces of each row per iteration)
-                        float4* st = reinterpret_cast<float4*>(const_cast<unsigned char*>(sb) + (k - KR) * 1024);
-                        st[0] = make_float4(e1[0], e1[1], e1[2], e1[3]);
-                        st[32] = make_float4(e1[4], e1[5], e1[6], e1[7]);
-                        if (!BONUS) {
-                            float4* sd = reinterpret_cast<float4*>(const_cast<unsigned char*>(sb) + kRowB + (k - KR) * 1024);
-                            sd[0] = make_float4(e2[0], e2[1], e2[2], e2[3]);
-                            sd[32] = make_float4(e2[4], e2[5], e2[6], e2[7]);
+                            et[k >= KH ? k - KH : 0][j] = e1[j];
+                            ed[k >= KH ? k - KH : 0][j] = e2[j];
                         }
                     }
                 }
             }
-            sB[0] = warp_sum(St.x + St.y);
-            sB[1] = warp_sum(Tt.x + Tt.y);
-            if (BONUS) {
-                sB[2] = sB[0];
-                sB[3] = sB[1];
-            } else {
-                sB[2] = warp_sum(Sd.x + Sd.y);
-                sB[3] = warp_sum(Td.x + Td.y);
-            }
+            if (K0 < KH) tmem_wait_st();            // the head is in tensor memory before anything reads it
         };
-        // The 2^t values of iteration k (compile-time k after unrolling): from registers, or from
-        // where pass B left them in the position's buffer.
+        // this warp's partial statistics of position n go to the control warp
+        auto publish = [&](bool bonus, int n) {
+            const float St = warp_sum(bSt.x + bSt.y), Tt = warp_sum(bTt.x + bTt.y);
+            float Sd = St, Td = Tt;
+            if (!bonus) {
+                Sd = warp_sum(bSd.x + bSd.y);
+                Td = warp_sum(bTd.x + bTd.y);
+            }
+            const float dz = warp_max_f32(bdz);
+            if (lane == 0) {
+                float4* w = reinterpret_cast<float4*>(&sh.wtab[n & 1][warp]);
+                const float Mt_w = (flags_w & 4u) ? kFloorL : -nmt_w * kLog2e;
+                const float Md_w = (flags_w & 8u) ? kFloorL : -nmd_w * kLog2e;
+                w[0] = make_float4(Mt_w, St, Tt, Md_w);
+                w[1] = make_float4(Sd, Td, __uint_as_float(flags_w & 3u), dz);
+                mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.entry_bar[n & 1]));
+            }
+            __syncwarp();
+        };
+        // all of pass B of one position, in two parts
+        auto b_head = [&](bool bonus, int n) {
+            if (bonus) pass_b(std::true_type{}, std::integral_constant<int, 0>{}, std::integral_constant<int, KH>{}, n);
+            else pass_b(std::false_type{}, std::integral_constant<int, 0>{}, std::integral_constant<int, KH>{}, n);
+        };
+        auto b_tail = [&](bool bonus, int n) {
+            if (bonus) pass_b(std::true_type{}, std::integral_constant<int, KH>{}, std::integral_constant<int, ITER>{}, n);
+            else pass_b(std::false_type{}, std::integral_constant<int, KH>{}, std::integral_constant<int, ITER>{}, n);
+        };
+
+        // The 2^t values of iteration k (compile-time k after unrolling): out of tensor memory
+        // (synchronously; the sampling scans and the vanilla residual use this) or from registers.
         auto load_kept = [&](int k, int n, bool with_d, float (&a)[8], float (&b)[8]) {
-            if (k < KR) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    a[j] = et[k < KR ? k : 0][j];
-                    b[j] = ed[k < KR ? k : 0][j];
-                }
-            } else {
-                const unsigned char* sb = buf_of(n);
-                const float4* st = reinterpret_cast<const float4*>(sb + (k - KR) * 1024);
-                const float4 a0 = st[0], a1 = st[32];
-                a[0] = a0.x, a[1] = a0.y, a[2] = a0.z, a[3] = a0.w, a[4] = a1.x, a[5] = a1.y, a[6] = a1.z, a[7] = a1.w;
+            if (k < KH) {
                 if (with_d) {
-                    const float4* sd = reinterpret_cast<const float4*>(sb + kRowB + (k - KR) * 1024);
-                    const float4 b0 = sd[0], b1 = sd[32];
-                    b[0] = b0.x, b[1] = b0.y, b[2] = b0.z, b[3] = b0.w, b[4] = b1.x, b[5] = b1.y, b[6] = b1.z, b[7] = b1.w;
+                    tmem_ld16(tm_of(n, k), a, b);
+                    tmem_wait_ld(a, b);
                 } else {
+                    tmem_ld8(tm_of(n, k), a);
+                    tmem_wait_ld(a);
 #pragma unroll
                     for (int j = 0; j < 8; ++j) b[j] = 0.f;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    a[j] = et[k >= KH ? k - KH : 0][j];
+                    b[j] = with_d ? ed[k >= KH ? k - KH : 0][j] : 0.f;
                 }
             }
         };
@@ -652,11 +799,73 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             return lastp;
         };
 
+        // ---- pass C (AdaSD mode) over the kept values of position n ---------------------------
+        // NEAR == false: A = sum (p+q) log2 (p+q) and the overlap indicator sum 2^t_p 2^t_q.
+        // NEAR == true (no logit of the two rows differs by more than kSNearDz): the divergence
+        // itself from non-negative terms, D_JS = 1/4 sum s phi(u) with s = p + q, u = (q - p) / s and
+        // phi(u) = (1-u) ln(1-u) + (1+u) ln(1+u) = u^2 + u^4/6 + u^6/15 + u^8/28 + ...; |u| <= tanh(1/2)
+        // there, so four terms are good to 5e-5 of phi, and nothing cancels however close the rows are.
+        // The loads of head iteration k + 1 are in flight while iteration k is worked on.
+        auto pass_c = [&](auto near_c, int n, float at, float ad, float& A, float& PQ) {
+            constexpr bool NEAR = decltype(near_c)::value;
+            float2 A2 = make_float2(0.f, 0.f), PQ2 = make_float2(0.f, 0.f);
+            const float2 at2 = make_float2(at, at), ad2 = make_float2(ad, ad);
+            const float2 tiny2 = make_float2(kTiny, kTiny), neg1 = make_float2(-1.f, -1.f);
+            auto body = [&](const float (&a)[8], const float (&d)[8]) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 a2 = make_float2(a[2 * j], a[2 * j + 1]);
+                    const float2 d2 = make_float2(d[2 * j], d[2 * j + 1]);
+                    const float2 pp = __ffma2_rn(a2, at2, tiny2);
+                    const float2 ss = __ffma2_rn(d2, ad2, pp);
+                    if (NEAR) {
+                        const float2 qq = __fmul2_rn(d2, ad2);
+                        const float2 df = __ffma2_rn(__fmul2_rn(a2, at2), neg1, qq);     // q - p
+                        const float2 u = __fmul2_rn(df, make_float2(rcp_approx(ss.x), rcp_approx(ss.y)));
+                        const float2 w = __fmul2_rn(u, u);
+                        float2 ph = __ffma2_rn(w, make_float2(1.f / 28.f, 1.f / 28.f), make_float2(1.f / 15.f, 1.f / 15.f));
+                        ph = __ffma2_rn(ph, w, make_float2(1.f / 6.f, 1.f / 6.f));
+                        ph = __ffma2_rn(ph, w, make_float2(1.f, 1.f));
+                        A2 = __ffma2_rn(__fmul2_rn(ss, w), ph, A2);
+                    } else {
+                        const float2 ll = make_float2(lg2(ss.x), lg2(ss.y));
+                        A2 = __ffma2_rn(ss, ll, A2);
+                        PQ2 = __ffma2_rn(a2, d2, PQ2);
+                    }
+                }
+            };
+            float xa[2][8], xd[2][8];              // head values in flight / in use
+            if (KH > 0 && k_on(0)) tmem_ld16(tm_of(n, 0), xa[0], xd[0]);
+#pragma unroll
+            for (int k = 0; k < ITER; ++k) {
+                if (k_on(k)) {
+                    if (k < KH) {
+                        tmem_wait_ld(xa[k & 1], xd[k & 1]);
+                        if (k + 1 < KH && k_on(k + 1)) tmem_ld16(tm_of(n, k + 1), xa[(k + 1) & 1], xd[(k + 1) & 1]);
+                        body(xa[k & 1], xd[k & 1]);
+                    } else {
+                        body(et[k >= KH ? k - KH : 0], ed[k >= KH ? k - KH : 0]);
+                    }
+                }
+            }
+            A = warp_sum(A2.x + A2.y);
+            PQ = NEAR ? 1.f : warp_sum(PQ2.x + PQ2.y);
+        };
+
         // ---------------------------------- main loop ----------------------------------------
+        // Invariant at the top of the loop: pass B of position n is complete and its partial
+        // statistics are with the control warp; the buffer of position n is being refilled.
         int n = 0;                 // sequence number of the current position
         if (pcx(0).pos < total) {
-            pass_a_any(pcx(0).bonus != 0, 0, true);
-            finish_a(pcx(0).bonus != 0);
+            const bool b0 = pcx(0).bonus != 0;
+            if (b0) pass_a(std::true_type{}, 0);
+            else pass_a(std::false_type{}, 0);
+            b_head(b0, 0);
+            b_tail(b0, 0);
+            publish(b0, 0);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            issue_pos(2);
         }
         while (pcx(n).pos < total) {
             const int par = n & 1;
@@ -665,29 +874,15 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const int npos = pcx(n + 1).pos;
             const bool nbonus = npos < total && pcx(n + 1).bonus != 0;
 
-            if (bonus) pass_b(std::true_type{}, n);
-            else pass_b(std::false_type{}, n);
-            if (lane == 0) {
-                float4* w = reinterpret_cast<float4*>(&sh.wtab[par][warp]);
-                const float Mt_w = (flags_w & 4u) ? kFloorL : -nmt_w * kLog2e;
-                const float Md_w = (flags_w & 8u) ? kFloorL : -nmd_w * kLog2e;
-                w[0] = make_float4(Mt_w, sB[0], sB[1], Md_w);
-                w[1] = make_float4(sB[2], sB[3], __uint_as_float(flags_w & 3u), 0.f);
-                mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.entry_bar[par]));
-            }
-            __syncwarp();
-            // while the control warps exchange the totals: maxima of the next position, if it
-            // has landed in the other buffer
-            bool a_fin = false;        // the next position's shifts are worked out already
+            // while the control warps exchange the totals of position n: maxima and the head of
+            // pass B of position n + 1 (its 2^t values go to the other half of tensor memory)
             if (npos < total) {
-                pass_a_any(nbonus, n + 1, false);
-                if (a_done) {          // nothing of position n needs this warp's shifts any more
-                    finish_a(nbonus);
-                    a_fin = true;
-                }
+                if (nbonus) pass_a(std::true_type{}, n + 1);
+                else pass_a(std::false_type{}, n + 1);
+                b_head(nbonus, n + 1);
             }
             wait_cta(&sh.scal_bar[par], ph);
-            const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft
+            const float4 m0 = *reinterpret_cast<const float4*>(&sh.wmsg[par][warp]);       // at, ad, ft, act
 
             // the target row's 2^t values of iteration k (what y_i ~ p_i is drawn from)
             auto vals_p = [&](int k, float(&v)[8]) {
@@ -696,31 +891,11 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             };
             float A = 0.f, PQ = 0.f;
             int tok = -1;
+            const int act = __float_as_int(m0.w);
             if (MODE == MODE_ADASD) {
-                // pass C: sum (p+q) log2 (p+q) and the overlap indicator sum 2^t_p 2^t_q
                 if (!bonus) {
-                    float2 A2 = make_float2(0.f, 0.f), PQ2 = make_float2(0.f, 0.f);
-                    const float2 at2 = make_float2(m0.x, m0.x), ad2 = make_float2(m0.y, m0.y);
-                    const float2 tiny2 = make_float2(kTiny, kTiny);
-#pragma unroll
-                    for (int k = 0; k < ITER; ++k) {
-                        if (k_on(k)) {
-                            float a[8], d[8];
-                            load_kept(k, n, true, a, d);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float2 a2 = make_float2(a[2 * j], a[2 * j + 1]);
-                                const float2 d2 = make_float2(d[2 * j], d[2 * j + 1]);
-                                const float2 pp = __ffma2_rn(a2, at2, tiny2);
-                                const float2 ss = __ffma2_rn(d2, ad2, pp);
-                                const float2 ll = make_float2(lg2(ss.x), lg2(ss.y));
-                                A2 = __ffma2_rn(ss, ll, A2);
-                                PQ2 = __ffma2_rn(a2, d2, PQ2);
-                            }
-                        }
-                    }
-                    A = warp_sum(A2.x + A2.y);
-                    PQ = warp_sum(PQ2.x + PQ2.y);
+                    if (act & 4) pass_c(std::true_type{}, n, m0.x, m0.y, A, PQ);
+                    else pass_c(std::false_type{}, n, m0.x, m0.y, A, PQ);
                 }
                 // y_i ~ p_i: the control warp says (a little later than the scale factors) whether
                 // this warp holds the crossing
@@ -730,7 +905,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             } else {
                 // vanilla: an accepted row needs nothing more; the bonus row draws from p; a rejected
                 // row draws from the residual max(0, p - q) / R, whose mass this warp now adds up
-                const int act = __float_as_int(m0.w);
                 const float at = m0.x, ad = m0.y;
                 auto vals_r = [&](int k, float(&v)[8]) {
                     float a[8], d[8];
@@ -763,11 +937,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     else if (sel == 2) tok = select_kept(m1.z, 1.f, m1.x, vals_r);
                 }
             }
-            // the buffer of position n is free: fetch position n + 2 into it (the bulk copy belongs
-            // to the async proxy and must come after this warp's own stores to the buffer)
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            issue_pos(n + 2);
             // this warp's sums (and the token, if it drew it) go to the leader CTA in one message
             if (lane == 0) {
                 const int fr = n & (kSFinRing - 1);
@@ -776,17 +945,21 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             }
             __syncwarp();
 
-            // the next position's maxima, if its copy had not landed during the exchange
-            if (npos < total && !a_fin) {
-                pass_a_any(nbonus, n + 1, true);
-                finish_a(nbonus);
+            // the rest of pass B of position n + 1 (its values stay in registers until pass C of
+            // n + 1), its partials to the control warp, and its buffer refilled with position n + 3
+            if (npos < total) {
+                b_tail(nbonus, n + 1);
+                publish(nbonus, n + 1);
+                // (the bulk copy belongs to the async proxy: order it after this warp's reads of the buffer)
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                issue_pos(n + 3);
             }
             ++n;
         }
         // a warp that gave up on a copy still waits (bounded) for whatever it had in flight
         if (!alive && nwu > 0) {
-            mbar_wait_bounded(bar_of(n), (uint32_t)(n >> 1) & 1u);
-            mbar_wait_bounded(bar_of(n + 1), (uint32_t)((n + 1) >> 1) & 1u);
+            for (int m = n_landed; m < n_issued; ++m) mbar_wait_bounded(bar_of(m), (uint32_t)(m >> 1) & 1u);
         }
     } else if (warp == kSCtl) {
         // ============================== control warp ======================================
@@ -860,12 +1033,13 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 const float St = warp_sum(ft * w0.y), Tt = warp_sum(ft * fmaf(dt, w0.y, w0.z));
                 const float Sd = warp_sum(fd * w1.x), Td = warp_sum(fd * fmaf(dd, w1.x, w1.y));
                 const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(w1.z));
+                const float dz = warp_max_f32(w1.w);          // largest |z_t - z_d| of this CTA's slice (>= 0)
                 if (lane == 0) mbar_expect_tx(reinterpret_cast<uint64_t*>(&sh.ctab_bar[par]), (uint32_t)(CS * 32));
                 if (lane < CS) {
                     const uint32_t dst = mapa_u32(&sh.ctab[par][rank], (uint32_t)lane);
                     const uint32_t bar = mapa_u32(&sh.ctab_bar[par], (uint32_t)lane);
                     st_async_v4(dst, make_float4(Mt, St, Tt, Md), bar);
-                    st_async_v4(dst + 16, make_float4(Sd, Td, __uint_as_float(fl), 0.f), bar);
+                    st_async_v4(dst + 16, make_float4(Sd, Td, __uint_as_float(fl), dz), bar);
                 }
             }
             // the row's totals from the CTA totals, lane c holding CTA c
@@ -885,9 +1059,11 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             // vanilla: alpha = min(1, p(x) / q(x)) at the draft token, and what is left to do
             const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(e1.z));
             const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL);
+            // AdaSD: the two rows are nearly equal everywhere -> pass C in its well-conditioned form
+            const bool near = (MODE == MODE_ADASD) && !bonus && !bad && (fl & 2u) && warp_max_f32(e1.w) <= kSNearDz;
             float alpha = 0.f;
             bool van_accept = true;
-            int act = 1;                          // AdaSD: every row draws y_i ~ p_i
+            int act = near ? 5 : 1;               // AdaSD: every row draws y_i ~ p_i
             if (MODE == MODE_VANILLA) {
                 if (!bonus) {
                     if (x_ok) {
@@ -959,7 +1135,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     }
                 }
             };
-            bool from_p = (act == 1);
+            bool from_p = ((act & 3) == 1);
             if (MODE == MODE_VANILLA && act == 2) {
                 // residual mass: warp sums -> CTA sum -> every CTA of the cluster
                 const uint32_t rph = nres & 1u;
@@ -992,6 +1168,13 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 f[6] = __uint_as_float(fl | (alive ? 0u : 1u));
                 f[7] = alpha;
                 f[8] = van_accept ? 1.f : 0.f;
+                f[9] = near ? 1.f : 0.f;
+            }
+            // every CTA's totals, for the finaliser's float64 combination
+            if (leader && lane < CS) {
+                float4* fc = reinterpret_cast<float4*>(&sh.finc[n & (kSFinRing - 1)][lane]);
+                fc[0] = e0;
+                fc[1] = e1;
             }
             __syncwarp();
             if (lane == 0) {
@@ -1033,17 +1216,23 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 wait_cta(&sh.c_bar[par], (uint32_t)(m / kSFinRing) & 1u);
                 const float4 c0 = sh.tabC[par][4 * lane], c1 = sh.tabC[par][4 * lane + 1];
                 const float4 c2 = sh.tabC[par][4 * lane + 2], c3 = sh.tabC[par][4 * lane + 3];
-                const float A = warp_sum(((c0.x + c1.x) + c2.x) + c3.x);
+                // The warps' sums are small numbers (1/72 of the total each): added up in float64, as
+                // are the CTAs' row statistics below.  In fp32 the totals (entropies of up to 17 bits)
+                // carry an error of about 1e-6 each, which the difference H(m) - (H(p)+H(q))/2 keeps.
+                const double A = warp_sum_f64(((double)c0.x + (double)c1.x) + ((double)c2.x + (double)c3.x));
                 const float PQ = warp_sum(((c0.y + c1.y) + c2.y) + c3.y);
                 const int tok_all = __reduce_max_sync(0xFFFFFFFFu, max(max(__float_as_int(c0.z), __float_as_int(c1.z)),
                                                                        max(__float_as_int(c2.z), __float_as_int(c3.z))));
+                const float Mt = sh.fin[par][0], Md = sh.fin[par][3];
+                FinOut fo = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                if (MODE == MODE_ADASD)
+                    fo = finalize_math(&sh.finc[par][0], CS, Mt, Md, A, PQ, __float_as_uint(sh.fin[par][6]),
+                                       sh.fin[par][9] != 0.f);
                 int done_b = -1;
                 if (lane == 0) {
                     const PosCtx& c = sh.pc[m & (kSPosRing - 1)];
                     const int b = c.pos / K1, i = c.pos - b * K1;
                     const bool bonus = c.bonus != 0;
-                    const float Mt = sh.fin[par][0], St = sh.fin[par][1], Tt = sh.fin[par][2];
-                    const float Md = sh.fin[par][3], Sd = sh.fin[par][4], Td = sh.fin[par][5];
                     const uint32_t fl = __float_as_uint(sh.fin[par][6]);
                     const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL) || !alive;
                     const size_t idt = (size_t)b * K1 + i, idd = (size_t)b * Kmax + i;
@@ -1059,9 +1248,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                         }
                         p.sc.van_tok[idt] = tok;
                     } else {
-                    const float lSt = lg2(St), lSd = lg2(Sd);
-                    const float Hbt = lSt - Tt / St, Hbd = lSd - Td / Sd;      // entropies in bits
-                    float Ht = kLn2 * Hbt, lse_t = kLn2 * (Mt + lSt);
+                    float Ht = fo.Ht, lse_t = fo.lse_t;
                     if (bad) Ht = lse_t = NAN;
                     p.sc.H_t[idt] = Ht;
                     p.sc.lse_t[idt] = lse_t;
@@ -1070,12 +1257,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     if (p.user.lse_t) p.user.lse_t[idt] = lse_t;
                     if (p.user.y) p.user.y[idt] = tok;
                     if (!bonus) {
-                        float Hd = kLn2 * Hbd, lse_d = kLn2 * (Md + lSd);
-                        // D_JS = H(m) - (H(p) + H(q)) / 2 with H(m) = (ln 2 / 2) (2 - sum s log2 s), s = p + q
-                        float jsd = 0.5f * kLn2 * ((2.f - A) - (Hbt + Hbd));
-                        jsd = (fl & 2u) ? fminf(fmaxf(jsd, 0.f), kLn2) : 0.f;   // identical rows: exactly 0
-                        if (!(PQ > 0.f)) jsd = kLn2;                            // disjoint supports: ln 2
-                        float dist = fminf(sqrtf(jsd / kLn2), 1.f);
+                        float Hd = fo.Hd, lse_d = fo.lse_d, jsd = fo.jsd, dist = fo.dist;
                         if (bad) Hd = lse_d = jsd = dist = NAN;
                         p.sc.H_d[idd] = Hd;
                         p.sc.lse_d[idd] = lse_d;
@@ -1213,7 +1395,9 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             }
         }
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     cluster.sync();   // no CTA leaves while a peer may still address its shared memory
+    if (warp == kSCtl) tmem_dealloc(tmem0, (uint32_t)kSTmemCols);   // by the warp that allocated it
 }
 
 }  // namespace adasd
