@@ -187,6 +187,7 @@ class Workload:
     adaptive_window: bool   # True: the entropy stop check sets K_t <= K each round
     vanilla: bool           # also run the vanilla comparison mode on the same inputs
     recipe: str
+    tau0: float = 0.0       # recipe "fixed_tau": the target noise of every position
 
     def scaled(self, **kw) -> "Workload":
         return replace(self, **kw)
@@ -207,6 +208,10 @@ class Workload:
             mid = 1.0 + 3.0 * param_uniform(self.seed, round_, B, K1, 1)
             s = np.where(sel < 0.1, 12.0, np.where(sel < 0.2, 0.2, mid))
             t = 0.05 + 3.95 * param_uniform(self.seed, round_, B, K1, 2)
+        elif self.recipe == "fixed_tau":
+            # nearly equal draft and target rows: the small-distance regime
+            s = 0.5 + 5.5 * param_uniform(self.seed, round_, B, K1, 0)
+            t = np.full((B, K1), self.tau0)
         elif self.recipe == "drift":
             s = 0.5 + 5.5 * param_uniform(self.seed, round_, B, K1, 0)
             frac = round_ / max(self.rounds - 1, 1)

@@ -157,6 +157,32 @@ def test_c5_streaming_adaptive_all_1024_rounds(torch):
     assert rep.rounds == 1024 and max(rep.window_hist) <= 16 and len(rep.window_hist) >= 4
 
 
+@pytest.mark.parametrize("V,dtype", [(128256, synth.BF16), (32000, synth.FP32)])
+@pytest.mark.parametrize("tau", [1e-3, 3e-3, 1e-2, 3e-2])
+def test_small_distance_regime_meets_the_plain_tolerance(torch, V, dtype, tau):
+    """Draft and target rows that nearly agree (target noise tau of 1e-3 .. 3e-2: distances of
+    3e-4 .. 2e-2, where d = sqrt(D_JS / ln 2) amplifies any error of D_JS): the kernels form
+    D_JS from non-negative terms there, and d must meet 1e-4 WITHOUT the widening that
+    tests/lockstep.py allows where fp32 cannot resolve D_JS."""
+    import json
+    import os
+    from tests.lockstep import Lockstep, TOL as LTOL
+    wl = synth.WORKLOADS["C3"].scaled(name=f"near_tau{tau:g}_V{V}", B=3, K=6, V=V, dtype=dtype, rounds=4,
+                                      recipe="fixed_tau", tau0=tau, vanilla=False)
+    ls = Lockstep(wl)
+    rep = ls.run()
+    s = rep.summary()
+    print(wl.name, s["max_err"])
+    log = os.environ.get("ADASD_PARITY_LOG")
+    if log:
+        with open(log, "a") as f:
+            f.write(json.dumps(dict(workload=wl.name, V=V, tau=tau, max_err_dist=s["max_err"]["dist"],
+                                    max_err_jsd=s["max_err"]["jsd"], dist_beyond_tol=s["dist_beyond_tol"])) + "\n")
+    assert rep.positions == 4 * 3 * 7
+    assert s["max_err"]["dist"] <= LTOL and rep.dist_beyond_tol == 0, s["max_err"]
+    assert s["max_err"]["jsd"] <= 1e-7, s["max_err"]
+
+
 def test_long_history_kde(torch):
     """Hundreds of rounds on a small vocabulary: long KDE lists, many rejections."""
     wl = synth.WORKLOADS["C3"].scaled(name="history", B=4, K=8, V=2048, rounds=300, vanilla=False)
