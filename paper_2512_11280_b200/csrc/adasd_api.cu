@@ -506,7 +506,10 @@ int adasd_create(adasd_ctx** out, const adasd_config* cfg) {
     ALLOC(t.van_tok, B * (K + 1));
     ALLOC(t.ticket, B);
     ALLOC(t.only_pos, B);
+    ALLOC(t.q_items, B);
+    ALLOC(t.q_ctl, 4);
 #undef ALLOC
+    if (rc == ADASD_OK && cudaMemset(t.q_items, 0xFF, B * sizeof(int32_t)) != cudaSuccess) rc = ADASD_ERR_CUDA;
     if (rc == ADASD_OK) fast_setup(c, prop.sharedMemPerBlockOptin);
     if (rc == ADASD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ADASD_ERR_CUDA;
     if (rc != ADASD_OK) {

@@ -25,6 +25,8 @@ struct Scratch {            // context-owned per-round scratch, all [B,Kmax(+1)]
     int32_t* van_tok;       // [B,Kmax+1] vanilla: resample (or bonus) candidate
     uint32_t* ticket;       // [B] arrival counter of a sequence's positions
     int32_t* only_pos;      // [B] vanilla: the position that is sampled (first rejection or bonus row)
+    int32_t* q_items;       // [B] chip-wide queue of completed sequences awaiting their tail (-1: empty)
+    uint32_t* q_ctl;        // [4] queue counters: pushed, drawn, workers gone (all 0 between launches)
 };
 
 struct VerifyParams {

@@ -62,7 +62,6 @@ static_assert(kSW % 4 == 0, "compute warps are spread evenly over the four lane 
 static_assert(kSW <= kCW, "the exchange tables are sized for kCW warps");
 constexpr float kSNearDz = 0.5f;                 // rows count as nearly equal when no logit differs by more
 constexpr int kSPosRing = 16;                    // positions the control warp keeps described
-constexpr int kSWorkQ = 16;                      // tail work queue entries per CTA
 constexpr int kSFinRing = 4;                     // positions whose sums may await finalisation
 constexpr uint32_t kSPollSpins = 1u << 24;       // polls of a progress counter before giving up
 
@@ -110,9 +109,7 @@ struct __align__(16) SpecShared {
     int32_t n_issued;                 // leader: positions whose messages have been sent
     int32_t n_final;                  // leader: number of positions of this cluster, -1 until known
     int32_t fin_done;                 // leader: positions finalised so far (written by the tail warp)
-    int32_t wq[kSWorkQ];              // non-leader: sequences whose tail this CTA's tail warp must run (-1: stop)
-    uint32_t wq_head, wq_tail;        // written by the leader's tail warp (remotely) / by this CTA's tail warp
-    float td[ADASD_KMAX_LIMIT], tH[ADASD_KMAX_LIMIT];   // tail warp scratch
+    float td[3][ADASD_KMAX_LIMIT], tH[3][ADASD_KMAX_LIMIT];   // scratch of the three tail workers of a CTA
 };
 
 // ---- mbarrier helpers with explicit scopes -----------------------------------------------
@@ -311,20 +308,39 @@ __device__ __forceinline__ void verify_tail_warp(const TailConfig& cfg, const Ta
                 di[k] = __shfl_sync(0xFFFFFFFFu, d, i);
                 ci[k] = __shfl_sync(0xFFFFFFFFu, cA, i);
             }
-            for (int j = lane; j < nA0; j += 32) {
-                const float xj = __ldcg(LA + j);
+            // four list entries per lane and trip, all four loads in flight together (the lists live
+            // in L2 / HBM: one load per trip would leave the warp waiting on memory, not on the
+            // special-function pipe); entries past the end sit far away, where the kernel is 0
+            for (int j0 = 0; j0 < nA0; j0 += 128) {
+                float xj[4];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float t = di[k] - xj;
-                    accA[k] += ex2(ci[k] * t * t);
+                for (int q = 0; q < 4; ++q) {
+                    const int j = j0 + 32 * q + lane;
+                    xj[q] = j < nA0 ? __ldcg(LA + j) : 1.0e9f;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const float t = di[k] - xj[q];
+                        accA[k] += ex2(ci[k] * t * t);
+                    }
                 }
             }
-            for (int j = lane; j < nR0; j += 32) {
-                const float xj = __ldcg(LR + j);
+            for (int j0 = 0; j0 < nR0; j0 += 128) {
+                float xj[4];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float t = di[k] - xj;
-                    accR[k] += ex2(cR * t * t);
+                for (int q = 0; q < 4; ++q) {
+                    const int j = j0 + 32 * q + lane;
+                    xj[q] = j < nR0 ? __ldcg(LR + j) : 1.0e9f;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const float t = di[k] - xj[q];
+                        accR[k] += ex2(cR * t * t);
+                    }
                 }
             }
 #pragma unroll
@@ -407,7 +423,6 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         sh.n_issued = 0;
         sh.n_final = -1;
         sh.fin_done = 0;
-        sh.wq_head = sh.wq_tail = 0u;
         for (int k = 0; k < 2; ++k) {
             mbar_init(reinterpret_cast<uint64_t*>(&sh.entry_bar[k]), kSW);
             mbar_init(reinterpret_cast<uint64_t*>(&sh.ctab_bar[k]), 1);
@@ -1279,32 +1294,17 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 return __shfl_sync(0xFFFFFFFFu, done_b, 0);
             };
 
-            // tails go round robin to the tail warps of the other CTAs of the cluster, which have
-            // nothing else to do: entry number k of CTA r's queue
-            uint32_t ndisp = 0;
-            auto send = [&](uint32_t r, uint32_t k, int b) {
+            // A completed sequence goes to the chip-wide queue of tails (device memory): whichever
+            // worker warp on the chip is free takes it.  (Handing the tails to this cluster's own
+            // workers would pile them up on the cluster that runs last, which draws most last tickets
+            // and would fall back further.)
+            auto push = [&](int b) {
                 if (lane == 0) {
-                    const uint32_t tail_addr = mapa_u32(&sh.wq_tail, r);
-                    bool room = !alive;
-                    for (uint32_t it = 0; !room && it < kSPollSpins; ++it) {
-                        room = (k - ld_cluster_u32(tail_addr)) < (uint32_t)kSWorkQ;
-                        if (!room) __nanosleep(100);
-                    }
-                    if (room) {
-                        __threadfence();
-                        st_cluster_u32(mapa_u32(&sh.wq[k % kSWorkQ], r), (uint32_t)b);
-                        fence_cluster();
-                        st_cluster_u32(mapa_u32(&sh.wq_head, r), k + 1u);
-                    } else {
-                        atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
-                    }
+                    __threadfence();                      // this sequence's position scalars are out
+                    const uint32_t idx = atomicAdd(p.sc.q_ctl + 0, 1u);
+                    if (idx < (uint32_t)p.B) *reinterpret_cast<volatile int32_t*>(p.sc.q_items + idx) = b;
                 }
                 __syncwarp();
-            };
-            auto dispatch = [&](int b) {
-                const uint32_t nw = (uint32_t)(CS - 1);
-                send(1u + ndisp % nw, ndisp / nw, b);
-                ++ndisp;
             };
             for (int m = 0;; ++m) {
                 // position m exists once its messages have gone out; the control warp says when
@@ -1340,11 +1340,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                             p.accept_len[done_b] = w;
                             p.next_token[done_b] = __ldcg(p.sc.van_tok + (size_t)done_b * K1 + w);
                         }
-                    } else if (CS > 1) {
-                        dispatch(done_b);
                     } else {
-                        __threadfence();
-                        verify_tail_warp(p.tail, io, p.st, done_b, sh.td, sh.tH);
+                        push(done_b);
                     }
                 }
                 if (lane == 0) {
@@ -1352,47 +1349,61 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     *reinterpret_cast<volatile int32_t*>(&sh.fin_done) = m + 1;
                 }
             }
-            // stop marks: CTA r has received the entries ndisp' < ndisp with ndisp' % nw == r - 1
-            for (uint32_t r = 1; r < (uint32_t)CS; ++r) {
-                const uint32_t nw = (uint32_t)(CS - 1);
-                const uint32_t sent = ndisp / nw + ((ndisp % nw) > (r - 1u) ? 1u : 0u);
-                send(r, sent, -1);
-            }
-        } else {
-            // worker: tails handed over by the leader's tail warp, in order, until the stop mark
-            TailIO io;
-            io.H_d = p.sc.H_d;
-            io.dist = p.sc.dist;
-            io.y = p.sc.y;
-            io.x = p.x;
-            io.u_accept = p.u_accept;
-            io.draft_len = p.draft_len;
-            io.p_acc = p.sc.p_acc;
-            io.p_acc_user = p.user.p_acc;
-            io.accept_len = p.accept_len;
-            io.next_token = p.next_token;
-            io.accept_len_rec = p.user.accept_len;
-            io.rejected_rec = p.user.rejected;
-            io.draft_len_rec = p.user.draft_len;
-            for (uint32_t k = 0;; ++k) {
-                int b = -2;
-                if (lane == 0) {
-                    for (uint32_t it = 0; it < kSPollSpins; ++it) {
-                        if (*reinterpret_cast<volatile uint32_t*>(&sh.wq_head) != k) {
-                            fence_cluster();
-                            b = *reinterpret_cast<volatile int32_t*>(&sh.wq[k % kSWorkQ]);
-                            break;
-                        }
-                        __nanosleep(200);
+        }
+    }
+    // ============================== tail workers ==========================================
+    // AdaSD mode: the tail warps of the non-leader CTAs and the two spare warps of every CTA take
+    // completed sequences from the chip-wide queue and run their tails (KDE/Bayes, accept scan,
+    // appends, T_G).  Every sequence has a bonus row, so exactly B tails are queued per launch: a
+    // worker leaves when it draws a number >= B, and the last worker to leave puts the counters
+    // back to zero for the next launch.
+    if (MODE == MODE_ADASD && warp >= kSTail && !(leader && warp == kSTail)) {
+        TailIO io;
+        io.H_d = p.sc.H_d;
+        io.dist = p.sc.dist;
+        io.y = p.sc.y;
+        io.x = p.x;
+        io.u_accept = p.u_accept;
+        io.draft_len = p.draft_len;
+        io.p_acc = p.sc.p_acc;
+        io.p_acc_user = p.user.p_acc;
+        io.accept_len = p.accept_len;
+        io.next_token = p.next_token;
+        io.accept_len_rec = p.user.accept_len;
+        io.rejected_rec = p.user.rejected;
+        io.draft_len_rec = p.user.draft_len;
+        const int slot = warp - kSTail;           // this worker's scratch
+        const uint32_t nworkers = (uint32_t)(gridDim.x / CS) * (uint32_t)(3 * CS - 1);
+        for (;;) {
+            int b = -2;
+            if (lane == 0) {
+                const uint32_t idx = atomicAdd(p.sc.q_ctl + 1, 1u);
+                if (idx >= (uint32_t)p.B) {
+                    b = -1;                       // no more tails this launch
+                    if (atomicAdd(p.sc.q_ctl + 2, 1u) + 1u == nworkers) {
+                        p.sc.q_ctl[0] = 0u;       // every worker has left: ready for the next launch
+                        p.sc.q_ctl[1] = 0u;
+                        p.sc.q_ctl[2] = 0u;
                     }
-                    if (b == -2) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                } else {
+                    volatile int32_t* item = p.sc.q_items + idx;
+                    for (uint32_t it = 0; it < kSPollSpins; ++it) {
+                        b = *item;
+                        if (b >= 0) break;
+                        __nanosleep(400);
+                    }
+                    if (b >= 0) *item = -1;       // the entry is free again
+                    else {
+                        b = -3;                   // nothing came: give this one up, go on
+                        atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
+                    }
                 }
-                b = __shfl_sync(0xFFFFFFFFu, b, 0);
-                if (b < 0) break;            // stop mark, or nothing ever came
-                __threadfence();
-                verify_tail_warp(p.tail, io, p.st, b, sh.td, sh.tH);
-                if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&sh.wq_tail) = k + 1u;
             }
+            b = __shfl_sync(0xFFFFFFFFu, b, 0);
+            if (b == -1) break;
+            if (b < 0) continue;
+            __threadfence();
+            verify_tail_warp(p.tail, io, p.st, b, sh.td[slot], sh.tH[slot]);
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
