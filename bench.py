@@ -286,7 +286,19 @@ def run_ours(args) -> dict:
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    ms, e2e_ms, verify_ms = max_over_ranks([ms, e2e_ms, verify_ms], dist, dev)
+    # the K draft calls of a round as one CUDA graph (issued one by one from Python the interpreter's
+    # time per call would be the measurement): microseconds per adasd_draft_entropy call
+    def drafts():
+        for s in range(nset):
+            for k in range(K):
+                ctx.draft_entropy(zd[s][:, k, :], Hk[k], u=u_d[s][k], token_out=tokk[k], stop_out=stopk[k],
+                                  draft_len=dlen, row_stride=K * V)
+    side = torch.cuda.Stream()
+    g_d = graph_of(torch, drafts, side)
+    time_replays(torch, g_d, 3, side)
+    draft_ms = time_replays(torch, g_d, 10, side) / (nset * K)
+
+    ms, e2e_ms, verify_ms, draft_ms = max_over_ranks([ms, e2e_ms, verify_ms, draft_ms], dist, dev)
 
     rows = step_rows(wl)
     rows_step = sum(rows.values())
@@ -309,6 +321,10 @@ def run_ours(args) -> dict:
                    "value_is": "rows read by adasd_verify / adasd_verify time (mean of the timed launches, max over ranks)",
                    "step_rows_per_s_all_calls": whole_job_rate(world, rows_step, args.steps, ms),
                    "kde_list_prefill": args.prefill,
+                   "draft_entropy": {"us_per_call": 1e3 * draft_ms, "bytes_per_call": B * row_bytes,
+                                     "gbs": B * row_bytes / (draft_ms * 1e-3) / 1e9,
+                                     "frac_of_peak": B * row_bytes / (draft_ms * 1e-3) / 1e9 / peak,
+                                     "timing": f"one CUDA graph of {nset * K} calls, 10 replays"},
                    "hbm_gbs_all_calls": world * rows_step * row_bytes * args.steps / (ms * 1e-3) / 1e9},
         "e2e": {"value": whole_job_rate(world, rows["verify"], e2e_steps, e2e_ms), "unit": UNIT,
                 "what": "pinned host logits -> device, adasd_verify through the C ABI, results -> host",
@@ -596,7 +612,14 @@ def run_adaptive_graph(args, torch, adasd, wl, rank, world, local, dev, dist) ->
     g2 = graph_of(torch, gen_only, side)
     t["gs"].round_dev.zero_()
     ms_gen = time_replays(torch, g2, R, side)
-    ms_round, ms_gen, verify_ms = max_over_ranks([ms_round, ms_gen, verify_ms], dist, dev)
+    def drafts():
+        for k in range(K):
+            t["ctx"].draft_entropy(t["zd"][:, k, :], t["Hk"][k], u=t["ud"][k], token_out=t["tokk"][k],
+                                   stop_out=t["stopk"][k], draft_len=t["dlen"], row_stride=K * V)
+    g3 = graph_of(torch, drafts, side)
+    time_replays(torch, g3, 3, side)
+    draft_ms = time_replays(torch, g3, 20, side) / K
+    ms_round, ms_gen, verify_ms, draft_ms = max_over_ranks([ms_round, ms_gen, verify_ms, draft_ms], dist, dev)
 
     # end to end: one round's logits from pinned host memory
     hd, ht = t["zd"].cpu().pin_memory(), t["zt"].cpu().pin_memory()
@@ -628,6 +651,10 @@ def run_adaptive_graph(args, torch, adasd, wl, rank, world, local, dev, dist) ->
              "generator_only_rounds_per_s": world * 1e3 / ms_gen, "generator_only_ms_per_round": ms_gen,
              "library_ms_per_round": ms_round - ms_gen,
              "mean_window": mean_kt, "mean_accept_len": mean_acc,
+             "draft_entropy": {"us_per_call": 1e3 * draft_ms, "bytes_per_call": B * wl.row_bytes,
+                               "gbs": B * wl.row_bytes / (draft_ms * 1e-3) / 1e9,
+                               "frac_of_peak": B * wl.row_bytes / (draft_ms * 1e-3) / 1e9 / measured_peak_gbs()[0],
+                               "timing": f"every row active: one CUDA graph of {K} calls, 20 replays"},
              "list_sizes_at_end": {"nE_max": int(nE.max()), "nA_max": int(nA.max()), "nR_max": int(nR.max())},
              "T_G_mean_at_end": float(T.mean()),
              "verify_sample": f"first {sample} rounds issued call by call, mean window {mean_kt_sample:.2f}",
