@@ -70,6 +70,12 @@ def lib():
     L.oracle_vanilla_round.argtypes = [_P, _P, _I, _I, C.c_int64, C.c_int64, _I, _P, _P, _D,
                                        _P, _P, _P, _P]
     L.oracle_vanilla_round.restype = None
+    L.oracle_argmax.argtypes = [_P, _I, _I]
+    L.oracle_argmax.restype = _I
+    L.oracle_greedy_round.argtypes = [_P, _I, _I, C.c_int64, _I, _P, _P, _P, _P]
+    L.oracle_greedy_round.restype = None
+    L.oracle_gen_only_update.argtypes = [_P, _P, _P, _P, _I, _I]
+    L.oracle_gen_only_update.restype = None
     return L
 
 
@@ -268,3 +274,29 @@ def vanilla_round(zd: np.ndarray, zt: np.ndarray, x, u_accept, u_resample: float
                                ua.ctypes.data, float(u_resample), alpha.ctypes.data,
                                C.byref(al), C.byref(nt), C.byref(mg))
     return dict(alpha=alpha, accept_len=al.value, next_token=nt.value, margin=mg.value)
+
+
+def argmax(z_row: np.ndarray) -> int:
+    """Most probable token of a raw logit row; lowest index among equal maxima."""
+    z, dt = _raw(z_row)
+    return lib().oracle_argmax(z.ctypes.data, dt, z.size)
+
+
+def greedy_round(zt: np.ndarray, x) -> dict:
+    """Greedy verification (Sec. 2.1.3) of the candidates x against target rows zt [>=K+1, V]."""
+    zt, dt = _raw(zt)
+    x = np.ascontiguousarray(x, dtype=np.int32)
+    K, V = x.size, zt.shape[-1]
+    assert zt.shape[0] >= K + 1
+    am = np.zeros(K + 1, dtype=np.int32)
+    al, nt = C.c_int32(), C.c_int32()
+    lib().oracle_greedy_round(zt.ctypes.data, dt, V, V, K, x.ctypes.data, am.ctypes.data, C.byref(al),
+                              C.byref(nt))
+    return dict(argmax=am, accept_len=al.value, next_token=nt.value)
+
+
+def gen_only_update(state: SequenceState, H_d, K_t: int, accept_len: int) -> None:
+    """Gen-Only feedback (Sec. 5): the rejected candidate's entropy joins L_E^R, T_G = mean."""
+    H = _f64(H_d)
+    lib().oracle_gen_only_update(state.LE.ctypes.data, C.byref(state.nE), C.byref(state.T_G),
+                                 H.ctypes.data, int(K_t), int(accept_len))

@@ -450,3 +450,75 @@ void oracle_vanilla_round(const void* zd, const void* zt, int32_t dtype, int32_t
     free(p);
     free(q);
 }
+
+/* ---------------------------------------------------------------- greedy decoding (Sec. 2.1.3) */
+
+/*
+ * The most probable token of a logit row, x = argmax_v z_v (Sec. 2.1.1, deterministic
+ * selection); among equal maxima the lowest index.  -1 for a row with NaN or without a
+ * finite logit.
+ */
+int32_t oracle_argmax(const void* z, int32_t dtype, int32_t V) {
+    double* zz = (double*)malloc(sizeof(double) * (size_t)V);
+    oracle_widen(z, dtype, V, zz);
+    int32_t best = -1;
+    double m = -INFINITY;
+    int bad = 0;
+    for (int32_t v = 0; v < V; ++v) {
+        if (isnan(zz[v])) bad = 1;
+        if (zz[v] > m) {
+            m = zz[v];
+            best = v;
+        }
+    }
+    free(zz);
+    return (bad || !isfinite(m)) ? -1 : best;
+}
+
+/*
+ * Greedy verification of one round for one sequence (Sec. 2.1.3, greedy decoding): the
+ * candidate x_i is accepted only if it equals the target's own choice argmax p_i; the scan
+ * stops at the first mismatch, and the token emitted after the accepted prefix is the
+ * target's choice at that position (the bonus row's if every candidate matched).
+ * argmax_out[K+1] receives the target's choices of the rows the scan looked at (-2 beyond).
+ */
+void oracle_greedy_round(const void* zt, int32_t dtype, int32_t V, int64_t t_row_stride, int32_t K,
+                         const int32_t* x, int32_t* argmax_out, int32_t* accept_len,
+                         int32_t* next_token) {
+    size_t esz = dtype == ORACLE_BF16 ? 2 : 4;
+    int32_t w = K;
+    for (int32_t i = 0; i <= K; ++i) argmax_out[i] = -2;
+    for (int32_t i = 0; i < K; ++i) {
+        argmax_out[i] = oracle_argmax((const char*)zt + (size_t)i * (size_t)t_row_stride * esz, dtype, V);
+        if (x[i] != argmax_out[i]) {
+            w = i;
+            break;
+        }
+    }
+    if (w == K)
+        argmax_out[K] = oracle_argmax((const char*)zt + (size_t)K * (size_t)t_row_stride * esz, dtype, V);
+    *accept_len = w;
+    *next_token = argmax_out[w];
+}
+
+/* ---------------------------------------------------------------- ablation variants (Sec. 5) */
+
+/*
+ * Gen-Only (Sec. 5, ablation): the generation component alone.  The draft loop stops on
+ * H(q_i) > T_G as in Alg. 1, verification is vanilla speculative sampling, and the feedback
+ * that T_G needs is the entropy of the rejected candidate: if vanilla verification rejected
+ * candidate accept_len (accept_len < K_t), H(q_{accept_len}) joins L_E^R and T_G becomes the
+ * mean of the list (Sec. 4.3).  No distances are collected.  H_d[K_t] are the entropies the
+ * draft steps produced.  (Verify-Only needs no function of its own: it is oracle_verify_round
+ * on a fixed window of five candidates.)
+ */
+void oracle_gen_only_update(double* LE, int32_t* nE, double* T_G, const double* H_d, int32_t K_t,
+                            int32_t accept_len) {
+    if (accept_len < 0 || accept_len >= K_t) return;          /* nothing was rejected */
+    if (!isfinite(H_d[accept_len])) return;
+    LE[*nE] = H_d[accept_len];
+    *nE += 1;
+    double s = 0.0;
+    for (int32_t j = 0; j < *nE; ++j) s += LE[j];
+    *T_G = s / (double)*nE;
+}

@@ -550,3 +550,69 @@ def test_vanilla_first_rejection_prefix():
     zt2[2, 3] -= 20.0                            # token 3 at position 2 becomes very unlikely
     out = oracle.vanilla_round(zd, zt2, [1, 2, 3, 4], [0.5] * K, 0.3)
     assert out["accept_len"] == 2 and out["next_token"] != 3 and np.isnan(out["alpha"][3])
+
+
+# ------------------------------------------------------------------ greedy decoding and the ablation variants
+
+def test_argmax_hand_cases_and_ties_take_the_lowest_index():
+    assert oracle.argmax(np.array([0.5, 2.0, -1.0, 2.0], dtype=np.float32)) == 1        # tie: lowest index
+    assert oracle.argmax(np.array([3.0, 2.0, -1.0, 2.5], dtype=np.float32)) == 0
+    assert oracle.argmax(np.array([-np.inf, -np.inf, -7.0, -np.inf], dtype=np.float32)) == 2
+    assert oracle.argmax(np.array([-np.inf] * 4, dtype=np.float32)) == -1
+    assert oracle.argmax(np.array([1.0, np.nan, 5.0, 0.0], dtype=np.float32)) == -1
+    # bf16 rounds 1.001 and 1.002 to the same value: a tie once widened, lowest index again
+    z = bf16_bits(np.array([0.0, 1.001, 1.002, 0.5]))
+    assert oracle.argmax(z) == 1
+    r = np.random.default_rng(3)
+    for V in (5, 1000, 128256):
+        z = r.normal(size=V).astype(np.float32)
+        assert oracle.argmax(z) == int(np.argmax(z))
+        p, _ = oracle.softmax(z.astype(np.float64))
+        assert oracle.argmax(z) == int(np.argmax(p))          # the most probable token (Sec. 2.1.1)
+
+
+def test_greedy_round_is_the_longest_matching_prefix():
+    """Sec. 2.1.3: accept x_i only if it equals argmax p_i; stop at the first mismatch; the
+    emitted token is the target's choice there (the bonus row's after a full match)."""
+    zt = np.array([[0.0, 3.0, 1.0, 2.0],      # argmax 1
+                   [5.0, 5.0, 1.0, 2.0],      # tie 0/1 -> 0
+                   [0.0, 1.0, 9.0, 2.0],      # 2
+                   [0.0, 1.0, 2.0, 7.0]],     # bonus row: 3
+                  dtype=np.float32)
+    o = oracle.greedy_round(zt, [1, 0, 2])                     # all match
+    assert (o["accept_len"], o["next_token"]) == (3, 3) and list(o["argmax"]) == [1, 0, 2, 3]
+    o = oracle.greedy_round(zt, [2, 0, 2])                     # fail at the first candidate
+    assert (o["accept_len"], o["next_token"]) == (0, 1) and list(o["argmax"]) == [1, -2, -2, -2]
+    o = oracle.greedy_round(zt, [1, 1, 2])                     # the tie goes to index 0, so 1 is a mismatch
+    assert (o["accept_len"], o["next_token"]) == (1, 0)
+    o = oracle.greedy_round(zt, [1, 0, 3])                     # fail at the last candidate
+    assert (o["accept_len"], o["next_token"]) == (2, 2)
+    o = oracle.greedy_round(zt[:1], [])                        # empty window: the bonus row decides
+    assert (o["accept_len"], o["next_token"]) == (0, 1)
+    # brute force on random small cases
+    r = np.random.default_rng(9)
+    for _ in range(200):
+        K, V = int(r.integers(1, 6)), 4
+        zt = r.integers(0, 3, size=(K + 1, V)).astype(np.float32)
+        x = r.integers(0, V, size=K)
+        am = [int(np.argmax(row)) for row in zt]
+        w = next((i for i in range(K) if x[i] != am[i]), K)
+        o = oracle.greedy_round(zt, x)
+        assert (o["accept_len"], o["next_token"]) == (w, am[w])
+
+
+def test_gen_only_feedback_is_the_running_mean_of_rejected_entropies():
+    """Sec. 5 (Gen-Only) with Sec. 4.3: only a rejection feeds T_G, with the entropy of the
+    rejected candidate; T_G is the mean of all of them; the distance lists stay empty."""
+    st = oracle.SequenceState(capacity=32)
+    H = [1.5, 0.25, 3.0, 2.0]
+    oracle.gen_only_update(st, H, 4, 4)                        # nothing rejected
+    assert st.nE.value == 0 and st.T_G.value == 0.0
+    oracle.gen_only_update(st, H, 4, 2)                        # candidate 2 rejected
+    assert st.nE.value == 1 and st.T_G.value == 3.0
+    oracle.gen_only_update(st, H, 4, 0)
+    assert st.nE.value == 2 and st.T_G.value == (3.0 + 1.5) / 2
+    oracle.gen_only_update(st, [np.nan, 1.0], 2, 0)            # an unusable row records nothing
+    assert st.nE.value == 2 and st.T_G.value == 2.25
+    oracle.gen_only_update(st, H, 2, 3)                        # accept_len beyond the window: ignored
+    assert st.nE.value == 2 and (st.nA.value, st.nR.value) == (0, 0)
