@@ -118,8 +118,10 @@ int adasd_reset(adasd_ctx* ctx, const int32_t* seq_ids_dev, int32_t n, void* str
  * One draft step for every active sequence (Algorithm 1, generation loop body;
  * Sec. 4.3; entropy as in Appendix A).  For row b of logits_dev [B,V]:
  *   H_out[b]   = H(q)             lse_out[b] = log-sum-exp (nullable)
- *   token_out[b] = inverse-CDF sample of q in index order with uniform u_dev[b]
- *                  (u_dev and token_out_dev nullable together: no sampling)
+ *   token_out[b] = inverse-CDF sample of q in index order with uniform u_dev[b];
+ *                  with u_dev NULL and token_out_dev given: the most probable token
+ *                  argmax q (greedy drafting, Sec. 2.1.3; lowest index among equal maxima);
+ *                  both NULL: no token
  *   stop_out[b]  = 1 iff H(q) > T_G[b]   (strict; the token stays in the window)
  *   draft_len_inout[b] += 1               (nullable)
  * active_inout_dev (nullable): rows with 0 are skipped and their outputs left
@@ -185,6 +187,39 @@ int adasd_vanilla_verify(adasd_ctx* ctx, const void* draft_logits_dev,
                          void* stream);
 
 /*
+ * Greedy verification of one round (Sec. 2.1.3, greedy decoding): candidate x_i is accepted
+ * only if it equals the target's own choice argmax p_i (lowest index among equal maxima); the
+ * scan stops at the first mismatch; next_token is the target's choice at that position, the
+ * bonus row's after a full match.  Only the target rows are read.  The adaptive state is
+ * neither read nor written.
+ *   target_logits_dev [B,Kmax+1,V], draft_tokens_dev [B,Kmax], draft_len_dev [B] (NULL: Kmax)
+ *   argmax_out_dev    [B,Kmax+1] nullable: the target's choices of rows 0..K_t
+ * A target row with NaN or without a finite logit has no choice (-1): it matches nothing and
+ * sets ADASD_STATUS_NAN.
+ */
+int adasd_greedy_verify(adasd_ctx* ctx, const void* target_logits_dev, int64_t t_seq_stride,
+                        int64_t t_row_stride, const int32_t* draft_tokens_dev,
+                        const int32_t* draft_len_dev, int32_t* accept_len_dev, int32_t* next_token_dev,
+                        int32_t* argmax_out_dev, void* stream);
+
+/*
+ * Feedback of the generation component on its own (Sec. 5, ablation variant "Gen-Only": the
+ * entropy stop check of Sec. 4.3 with vanilla verification).  Where vanilla verification
+ * rejected a candidate (accept_len[b] < draft_len[b]) the entropy H(q) of that candidate, as
+ * adasd_draft_entropy reported it, joins L_E^R and T_G[b] becomes the mean of the list; the
+ * distance lists are not touched.  H_draft_dev [B,Kmax]: entropy of draft step i of sequence b.
+ *
+ * The paper's variants as sequences of calls:
+ *   AdaSD        draft_entropy (stop on H > T_G) ... ; verify (ADASD_FUSE_UPDATE)
+ *   Gen-Only     draft_entropy (stop on H > T_G) ... ; vanilla_verify ; gen_only_update
+ *   Verify-Only  five draft_entropy calls, stop flags ignored ; verify (ADASD_FUSE_UPDATE)
+ *   Vanilla      five draft_entropy calls ; vanilla_verify
+ *   greedy       draft_entropy with u_dev = NULL (argmax q) ... ; greedy_verify
+ */
+int adasd_gen_only_update(adasd_ctx* ctx, const float* H_draft_dev, const int32_t* draft_len_dev,
+                          const int32_t* accept_len_dev, void* stream);
+
+/*
  * Vanilla verification for callers that must not allocate device memory.  (The paper has
  * no counterpart: this is a packaging variant of adasd_vanilla_verify, same inputs, same
  * outputs, same arithmetic.)
@@ -238,6 +273,20 @@ int adasd_get_thresholds(adasd_ctx* ctx, float* T_G_dev, int32_t* nE_dev, int32_
  */
 int adasd_state_export(adasd_ctx* ctx, int32_t seq, void* host_buf, size_t* bytes);
 int adasd_state_import(adasd_ctx* ctx, int32_t seq, const void* host_buf, size_t bytes);
+
+/*
+ * Self-test of the failure detection of the device code (the paper has no counterpart).  Every
+ * wait in the kernels is bounded: a warp whose wait runs out sets ADASD_STATUS_TIMEOUT, stops
+ * waiting and copying, publishes NaN / -1 for what it could not compute and lets the kernel
+ * end.  This call runs one draft step (as adasd_draft_entropy with no active mask) in which
+ * one warp working on row `row` never asks for its first chunk of the row and waits for it
+ * only briefly: the wait runs out with nothing in flight.  Afterwards adasd_status() reports
+ * ADASD_STATUS_TIMEOUT, H_out[row] is NaN and token_out[row] is -1, every other row is as
+ * usual, and the context is fit for further calls.  Needs the streaming draft kernel (bf16
+ * rows of a multiple of 8 logits, V >= 8192, 16-byte aligned), else ADASD_ERR_SHAPE.
+ */
+int adasd_selftest_expired_wait(adasd_ctx* ctx, const void* logits_dev, int64_t row_stride, int32_t row,
+                                const float* u_dev, float* H_out_dev, int32_t* token_out_dev, void* stream);
 
 /* Reads and clears the sticky status word (ADASD_STATUS_* bits).  Synchronises. */
 int adasd_status(adasd_ctx* ctx, uint32_t* status_out);

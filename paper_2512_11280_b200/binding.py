@@ -64,6 +64,9 @@ def lib() -> C.CDLL:
         "adasd_vanilla_verify": [P, P, P, I64, I64, I64, I64, P, P, P, P, P, P, P, P],
         "adasd_vanilla_verify_static": [I32, I32, I32, I32, P, P, I64, I64, I64, I64, P, P, P, P,
                                         P, P, P, P, P],
+        "adasd_greedy_verify": [P, P, I64, I64, P, P, P, P, P, P],
+        "adasd_gen_only_update": [P, P, P, P, P],
+        "adasd_selftest_expired_wait": [P, P, I64, I32, P, P, P, P],
         "adasd_get_thresholds": [P, P, P, P, P, P],
         "adasd_state_export": [P, I32, P, C.POINTER(C.c_size_t)],
         "adasd_state_import": [P, I32, P, C.c_size_t],
@@ -144,6 +147,21 @@ def adasd_vanilla_verify_static(B, V, Kmax, dtype, draft_logits_dev, target_logi
                                              draft_len_dev, u_accept_dev, u_resample_dev,
                                              accept_len_dev, next_token_dev, alpha_out_dev,
                                              status_out_dev, stream)
+
+
+def adasd_greedy_verify(ctx, target_logits_dev, t_seq_stride, t_row_stride, draft_tokens_dev,
+                        draft_len_dev, accept_len_dev, next_token_dev, argmax_out_dev, stream) -> int:
+    return lib().adasd_greedy_verify(ctx, target_logits_dev, t_seq_stride, t_row_stride, draft_tokens_dev,
+                                     draft_len_dev, accept_len_dev, next_token_dev, argmax_out_dev, stream)
+
+
+def adasd_gen_only_update(ctx, H_draft_dev, draft_len_dev, accept_len_dev, stream) -> int:
+    return lib().adasd_gen_only_update(ctx, H_draft_dev, draft_len_dev, accept_len_dev, stream)
+
+
+def adasd_selftest_expired_wait(ctx, logits_dev, row_stride, row, u_dev, H_out_dev, token_out_dev, stream) -> int:
+    return lib().adasd_selftest_expired_wait(ctx, logits_dev, row_stride, row, u_dev, H_out_dev, token_out_dev,
+                                             stream)
 
 
 def adasd_get_thresholds(ctx, T_G_dev, nE_dev, nA_dev, nR_dev, stream) -> int:
@@ -263,6 +281,17 @@ class Context:
                                          _ptr(draft_len), u_accept.data_ptr(), u_resample.data_ptr(),
                                          accept_len.data_ptr(), next_token.data_ptr(),
                                          _ptr(alpha_out), self._stream()), "adasd_vanilla_verify")
+
+    def greedy_verify(self, target_logits, draft_tokens, accept_len, next_token, draft_len=None,
+                      argmax_out=None) -> None:
+        self._check(adasd_greedy_verify(self.handle, target_logits.data_ptr(), target_logits.stride(0),
+                                        target_logits.stride(1), draft_tokens.data_ptr(), _ptr(draft_len),
+                                        accept_len.data_ptr(), next_token.data_ptr(), _ptr(argmax_out),
+                                        self._stream()), "adasd_greedy_verify")
+
+    def gen_only_update(self, H_draft, accept_len, draft_len=None) -> None:
+        self._check(adasd_gen_only_update(self.handle, H_draft.data_ptr(), _ptr(draft_len),
+                                          accept_len.data_ptr(), self._stream()), "adasd_gen_only_update")
 
     def get_thresholds(self):
         """(T_G, nE, nA, nR) as new device tensors."""

@@ -15,6 +15,7 @@
 #include "adasd_spec.cuh"
 #include "adasd_draft.cuh"
 #include "adasd_vanilla.cuh"
+#include "adasd_modes.cuh"
 
 using namespace adasd;
 
@@ -381,6 +382,22 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
                : launch_cluster(verify_kernel<float, false, MODE>, p, positions, cs, stream);
 }
 
+// The most probable token of every needed row (greedy drafting and greedy verification).
+int launch_argmax(adasd_ctx* ctx, const ArgmaxParams& a, cudaStream_t stream) {
+    const long long rows = (long long)a.B * a.R;
+    const unsigned grid = (unsigned)std::min<long long>(rows, 4LL * ctx->sm_count);
+    const bool vec = vec_ok(a.z, ctx->cfg.dtype, {a.seq_stride, a.row_stride});
+    if (ctx->cfg.dtype == ADASD_BF16) {
+        if (vec) row_argmax_kernel<__nv_bfloat16, true><<<grid, kAThreads, 0, stream>>>(a);
+        else row_argmax_kernel<__nv_bfloat16, false><<<grid, kAThreads, 0, stream>>>(a);
+    } else {
+        if (vec) row_argmax_kernel<float, true><<<grid, kAThreads, 0, stream>>>(a);
+        else row_argmax_kernel<float, false><<<grid, kAThreads, 0, stream>>>(a);
+    }
+    CUDA_TRY(cudaGetLastError());
+    return ADASD_OK;
+}
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = false;
@@ -545,12 +562,13 @@ int adasd_reset(adasd_ctx* ctx, const int32_t* seq_ids_dev, int32_t n, void* str
     return ADASD_OK;
 }
 
-int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stride,
-                        const float* u_dev, uint8_t* active_inout_dev, float* H_out_dev,
-                        float* lse_out_dev, int32_t* token_out_dev, uint8_t* stop_out_dev,
-                        int32_t* draft_len_inout_dev, void* stream) {
+// adasd_draft_entropy, optionally (expire_row >= 0) as the self-test of the bounded waits
+static int draft_entropy_impl(adasd_ctx* ctx, const void* logits_dev, int64_t row_stride,
+                              const float* u_dev, uint8_t* active_inout_dev, float* H_out_dev,
+                              float* lse_out_dev, int32_t* token_out_dev, uint8_t* stop_out_dev,
+                              int32_t* draft_len_inout_dev, void* stream, int32_t expire_row) {
     if (!ctx || !logits_dev || !H_out_dev) return ADASD_ERR_NULL;
-    if ((u_dev == nullptr) != (token_out_dev == nullptr)) return ADASD_ERR_NULL;
+    if (u_dev != nullptr && token_out_dev == nullptr) return ADASD_ERR_NULL;
     if (int rc = check_device(ctx)) return rc;
     if (!aligned_to(logits_dev, elt_size(ctx->cfg.dtype)) ||
         !aligned4({u_dev, H_out_dev, lse_out_dev, token_out_dev, draft_len_inout_dev}))
@@ -564,15 +582,34 @@ int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stri
     p.active = active_inout_dev;
     p.H_out = H_out_dev;
     p.lse_out = lse_out_dev;
-    p.token_out = token_out_dev;
+    p.token_out = u_dev ? token_out_dev : nullptr;
     p.stop_out = stop_out_dev;
     p.draft_len = draft_len_inout_dev;
     p.st = ctx->st;
     p.B = ctx->cfg.B;
     p.V = ctx->cfg.V;
+    p.expire_row = expire_row;
     const int cs = pick_cluster(ctx, p.B);
     const bool vec = vec_ok(logits_dev, ctx->cfg.dtype, {row_stride});
+    if (expire_row >= 0 && !(vec && ctx->draft_stream && expire_row < ctx->cfg.B))
+        return ADASD_ERR_SHAPE;                  // the self-test needs the streaming kernel
     cudaStream_t st = (cudaStream_t)stream;
+    if (!u_dev && token_out_dev) {
+        // greedy drafting: the most probable token of every active row, before the step below can
+        // clear a row's entry in the active mask (the token that trips the stop check stays)
+        ArgmaxParams a;
+        memset(&a, 0, sizeof(a));
+        a.z = logits_dev;
+        a.seq_stride = row_stride;
+        a.row_stride = 0;
+        a.active = active_inout_dev;
+        a.out = token_out_dev;
+        a.status = ctx->st.status;
+        a.B = ctx->cfg.B;
+        a.R = 1;
+        a.V = ctx->cfg.V;
+        if (int rc = launch_argmax(ctx, a, st)) return rc;
+    }
     if (vec && ctx->draft_stream) {
         const int P = draft_stream_p(ctx);
         // a grid of at most one CTA per SM runs 16 warps per CTA, a larger one 8 (two CTAs per SM)
@@ -607,6 +644,21 @@ int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stri
                    : launch_cluster(draft_kernel<__nv_bfloat16, false>, p, p.B, cs, st);
     return vec ? launch_cluster(draft_kernel<float, true>, p, p.B, cs, st)
                : launch_cluster(draft_kernel<float, false>, p, p.B, cs, st);
+}
+
+int adasd_draft_entropy(adasd_ctx* ctx, const void* logits_dev, int64_t row_stride,
+                        const float* u_dev, uint8_t* active_inout_dev, float* H_out_dev,
+                        float* lse_out_dev, int32_t* token_out_dev, uint8_t* stop_out_dev,
+                        int32_t* draft_len_inout_dev, void* stream) {
+    return draft_entropy_impl(ctx, logits_dev, row_stride, u_dev, active_inout_dev, H_out_dev, lse_out_dev,
+                              token_out_dev, stop_out_dev, draft_len_inout_dev, stream, -1);
+}
+
+int adasd_selftest_expired_wait(adasd_ctx* ctx, const void* logits_dev, int64_t row_stride, int32_t row,
+                                const float* u_dev, float* H_out_dev, int32_t* token_out_dev, void* stream) {
+    if (row < 0) return ADASD_ERR_SHAPE;
+    return draft_entropy_impl(ctx, logits_dev, row_stride, u_dev, nullptr, H_out_dev, nullptr, token_out_dev,
+                              nullptr, nullptr, stream, row);
 }
 
 int adasd_verify(adasd_ctx* ctx, const void* draft_logits_dev, const void* target_logits_dev,
@@ -674,6 +726,49 @@ int adasd_vanilla_verify(adasd_ctx* ctx, const void* draft_logits_dev,
     p.next_token = next_token_dev;
     p.alpha_out = alpha_out_dev;
     return launch_verify<MODE_VANILLA>(ctx, p, (cudaStream_t)stream);
+}
+
+int adasd_greedy_verify(adasd_ctx* ctx, const void* target_logits_dev, int64_t t_seq_stride,
+                        int64_t t_row_stride, const int32_t* draft_tokens_dev,
+                        const int32_t* draft_len_dev, int32_t* accept_len_dev, int32_t* next_token_dev,
+                        int32_t* argmax_out_dev, void* stream) {
+    if (!ctx || !target_logits_dev || !draft_tokens_dev || !accept_len_dev || !next_token_dev)
+        return ADASD_ERR_NULL;
+    if (int rc = check_device(ctx)) return rc;
+    if (!aligned_to(target_logits_dev, elt_size(ctx->cfg.dtype)) ||
+        !aligned4({draft_tokens_dev, draft_len_dev, accept_len_dev, next_token_dev, argmax_out_dev}))
+        return ADASD_ERR_ALIGN;
+    if (int rc = check_strides(ctx, t_seq_stride, t_row_stride)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = ctx->cfg.B, K = ctx->cfg.Kmax;
+    ArgmaxParams a;
+    memset(&a, 0, sizeof(a));
+    a.z = target_logits_dev;
+    a.seq_stride = t_seq_stride;
+    a.row_stride = t_row_stride;
+    a.draft_len = draft_len_dev;
+    a.out = ctx->sc.van_tok;                 // [B, Kmax + 1] scratch of the comparison modes
+    a.status = ctx->st.status;
+    a.B = B;
+    a.R = K + 1;
+    a.V = ctx->cfg.V;
+    if (int rc = launch_argmax(ctx, a, st)) return rc;
+    greedy_accept_kernel<<<(B + 127) / 128, 128, 0, st>>>(draft_tokens_dev, ctx->sc.van_tok, draft_len_dev,
+                                                        accept_len_dev, next_token_dev, argmax_out_dev, B, K);
+    CUDA_TRY(cudaGetLastError());
+    return ADASD_OK;
+}
+
+int adasd_gen_only_update(adasd_ctx* ctx, const float* H_draft_dev, const int32_t* draft_len_dev,
+                          const int32_t* accept_len_dev, void* stream) {
+    if (!ctx || !H_draft_dev || !accept_len_dev) return ADASD_ERR_NULL;
+    if (int rc = check_device(ctx)) return rc;
+    if (!aligned4({H_draft_dev, draft_len_dev, accept_len_dev})) return ADASD_ERR_ALIGN;
+    const int B = ctx->cfg.B;
+    gen_only_update_kernel<<<(B + 127) / 128, 128, 0, (cudaStream_t)stream>>>(ctx->st, H_draft_dev, draft_len_dev,
+                                                                             accept_len_dev, B, ctx->cfg.Kmax);
+    CUDA_TRY(cudaGetLastError());
+    return ADASD_OK;
 }
 
 int adasd_get_thresholds(adasd_ctx* ctx, float* T_G_dev, int32_t* nE_dev, int32_t* nA_dev,

@@ -53,8 +53,8 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint64_t* bar, uint32_t parit
     return ok;
 }
 // Bounded wait: false if the copy did not complete within the spin budget.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kCWaitSpins; ++it)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t spins = kCWaitSpins) {
+    for (uint32_t it = 0; it < spins; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

@@ -73,8 +73,11 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
     // writes to itself, and every warp waits on barriers it set up itself)
     if (P > 1) cluster.sync();
     bool alive = true;
+    // self-test of the give-up path: this warp never asks for its first chunk and waits for it only
+    // briefly, so the wait runs out with nothing in flight
+    const bool expiring = (b == p.expire_row && rank == 0 && warp == 0);
     auto issue = [&](int c) {
-        if (lane == 0 && c < nch) {
+        if (lane == 0 && c < nch && !(expiring && c == 0)) {
             const uint32_t bytes = (uint32_t)min(kDChunkUnits, nwu - c * kDChunkUnits) * 16u;
             uint64_t* bar = reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]);
             mbar_expect_tx(bar, bytes);
@@ -96,13 +99,16 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
             r0->cm[rank * kDW + warp][lane] = kFloorL;
             r0->cs[rank * kDW + warp][lane] = 0.f;
         }
+        int cfail = -1;                                      // chunk whose copy never landed
         for (int c = 0; c < nch; ++c) {
-            bool ok = alive && mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u);
+            bool ok = alive && mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u,
+                                                 expiring && c == 0 ? 64u : kCWaitSpins);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) {
                 if (alive && lane == 0) atomicOr(p.st.status, ADASD_STATUS_TIMEOUT);
                 alive = false;
                 bad = 1u;
+                cfail = c;
                 break;
             }
             const unsigned char* sb = bufs + (size_t)(c & 1) * kDChunkBytes + (size_t)lane * 16;
@@ -153,6 +159,13 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
                 r0->cm[rank * kDW + warp][c] = M;
                 r0->cs[rank * kDW + warp][c] = cs;
             }
+        }
+        // a warp that gave up still waits (bounded) for what it had asked for and not taken: the
+        // chunk it gave up on and the one after it; nothing may land in this CTA after it has gone
+        if (cfail >= 0) {
+            for (int c = cfail; c < min(cfail + 2, nch); ++c)
+                if (!(expiring && c == 0))
+                    mbar_wait_bounded(reinterpret_cast<uint64_t*>(&sh.bar[warp][c & 1]), (uint32_t)(c >> 1) & 1u);
         }
         const float Sw = warp_sum(S2.x + S2.y), Tw = warp_sum(T2.x + T2.y);
         bad = __reduce_or_sync(0xFFFFFFFFu, bad);

@@ -60,6 +60,7 @@ struct DraftParams {
     int32_t* draft_len;
     State st;
     int32_t B, V;
+    int32_t expire_row;     // self-test of the bounded waits: the row whose first copy is never asked for (-1: none)
 };
 
 struct RowShared {
