@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_HERE, "libadasd_oracle.so")
 _SRC = os.path.join(_HERE, "adasd_oracle.c")
 
-BF16, FP32 = 0, 1
+BF16, FP32, F64 = 0, 1, 2
 LN2 = math.log(2.0)
 
 
@@ -76,6 +76,8 @@ def lib():
     L.oracle_greedy_round.restype = None
     L.oracle_gen_only_update.argtypes = [_P, _P, _P, _P, _I, _I]
     L.oracle_gen_only_update.restype = None
+    L.oracle_warp_logits.argtypes = [_P, _I, _D, _I, _D, _P, _P]
+    L.oracle_warp_logits.restype = None
     return L
 
 
@@ -93,13 +95,16 @@ def _f64(a) -> np.ndarray:
 
 
 def _raw(z: np.ndarray):
-    """(contiguous array, dtype code) for bf16-bit (uint16) or float32 logits."""
+    """(contiguous array, dtype code) for bf16-bit (uint16) or float32 logits, or for float64
+    rows that `warp` returned."""
     z = np.ascontiguousarray(z)
     if z.dtype == np.uint16:
         return z, BF16
     if z.dtype == np.float32:
         return z, FP32
-    raise TypeError("logits must be uint16 (bf16 bits) or float32")
+    if z.dtype == np.float64:
+        return z, F64
+    raise TypeError("logits must be uint16 (bf16 bits), float32 or float64 (warped rows)")
 
 
 # ----------------------------------------------------------------------------- definitions
@@ -109,6 +114,22 @@ def widen(z: np.ndarray) -> np.ndarray:
     out = np.empty(z.shape, dtype=np.float64)
     lib().oracle_widen(z.ctypes.data, dt, z.size, out.ctypes.data)
     return out
+
+
+def warp(z: np.ndarray, temperature: float = 1.0, top_k: int = 0, top_p: float = 1.0) -> tuple:
+    """Adjusted distribution of Sec. 2.1.1 as logits (float64, -inf where a token is cut), for
+    one row or a stack of rows; also the smallest top-p decision margin over the rows."""
+    zz = widen(z) if z.dtype != np.float64 else np.ascontiguousarray(z)
+    V = zz.shape[-1]
+    flat = zz.reshape(-1, V)
+    out = np.empty_like(flat)
+    margin = math.inf
+    for r in range(flat.shape[0]):
+        m = _D(0.0)
+        lib().oracle_warp_logits(flat[r].ctypes.data, V, float(temperature), int(top_k), float(top_p),
+                                 out[r].ctypes.data, C.byref(m))
+        margin = min(margin, m.value)
+    return out.reshape(zz.shape), margin
 
 
 def softmax(z) -> tuple:

@@ -14,7 +14,9 @@
  * the two printed forms of the JS divergence, KL = CE - H, triangle inequality of
  * the JS distance, hand-derived V=4 values, brute-force inverse CDF, Leviathan's
  * output-law identity for the vanilla mode, KDE against quadrature and library
- * routines, running-mean threshold trajectories.
+ * routines, running-mean threshold trajectories; the adjusted distribution (temperature,
+ * top-k, top-p) against a hand-derived V=8 row, p^(1/T), a partition, an independent
+ * sort-and-cumsum rule and its minimality.
  *
  * Parity unpinned (the paper does not fix them; the readings are listed in the
  * design notes): the KDE kernel and bandwidth rule, the cold-start rule for the
@@ -28,6 +30,9 @@
 
 #define ORACLE_BF16 0
 #define ORACLE_FP32 1
+#define ORACLE_F64 2   /* rows already in double: the output of oracle_warp_logits */
+
+static size_t elt_size(int32_t dtype) { return dtype == ORACLE_BF16 ? 2 : dtype == ORACLE_FP32 ? 4 : 8; }
 
 /* ---------------------------------------------------------------- input widening */
 
@@ -40,9 +45,11 @@ void oracle_widen(const void* z, int32_t dtype, int64_t n, double* out) {
             c.u = (uint32_t)h[i] << 16;
             out[i] = (double)c.f;
         }
-    } else {
+    } else if (dtype == ORACLE_FP32) {
         const float* f = (const float*)z;
         for (int64_t i = 0; i < n; ++i) out[i] = (double)f[i];
+    } else {
+        memcpy(out, z, sizeof(double) * (size_t)n);
     }
 }
 
@@ -199,6 +206,78 @@ int32_t oracle_inv_cdf(const double* p, int32_t V, double u, double* margin_out)
     return last_pos;
 }
 
+/* ---------------------------------------------------------------- adjusted distribution */
+
+typedef struct { double z; int32_t v; } warp_item;
+static int warp_desc(const void* a, const void* b) {
+    const warp_item* x = (const warp_item*)a;
+    const warp_item* y = (const warp_item*)b;
+    if (x->z > y->z) return -1;
+    if (x->z < y->z) return 1;
+    return (x->v > y->v) - (x->v < y->v);
+}
+
+/*
+ * The adjusted distribution a token is sampled from (Sec. 2.1.1: temperature scaling,
+ * top-k sampling, top-p sampling), as logits: out_v = z_v / temperature for the tokens
+ * that stay, -inf for the tokens that are cut, applied in that order.
+ *
+ *   temperature > 0        z_v / temperature.
+ *   0 < top_k < V          the k most probable tokens stay; tokens whose logit equals the
+ *                          k-th largest stay with it (a tie is never split).
+ *   0 < top_p < 1          with pi = softmax of what the first two steps left, a token
+ *                          stays iff the tokens STRICTLY more probable than it hold less
+ *                          than top_p of the mass: the smallest set of most probable
+ *                          tokens whose mass reaches top_p, ties at its edge included.
+ *   top_k <= 0 or >= V, top_p >= 1, temperature == 1: that step changes nothing.
+ *
+ * margin_out: the smallest |mass of the strictly more probable tokens - top_p| over the
+ * groups of equally probable tokens, i.e. how close the top-p decision came to going the
+ * other way (+inf when top-p is off).  A row with NaN or without a finite logit is
+ * returned scaled and uncut.
+ */
+void oracle_warp_logits(const double* z, int32_t V, double temperature, int32_t top_k, double top_p,
+                        double* out, double* margin_out) {
+    *margin_out = INFINITY;
+    int bad = 0, finite = 0;
+    for (int32_t v = 0; v < V; ++v) {
+        out[v] = z[v] / temperature;
+        if (isnan(z[v])) bad = 1;
+        if (isfinite(z[v])) finite = 1;
+        if (z[v] == INFINITY) bad = 1;
+    }
+    if (bad || !finite) return;
+    warp_item* it = (warp_item*)malloc(sizeof(warp_item) * (size_t)V);
+    if (top_k > 0 && top_k < V) {
+        for (int32_t v = 0; v < V; ++v) { it[v].z = out[v]; it[v].v = v; }
+        qsort(it, (size_t)V, sizeof(warp_item), warp_desc);
+        const double kth = it[top_k - 1].z;
+        for (int32_t v = 0; v < V; ++v)
+            if (out[v] < kth) out[v] = -INFINITY;
+    }
+    if (top_p > 0.0 && top_p < 1.0) {
+        double* pi = (double*)malloc(sizeof(double) * (size_t)V);
+        oracle_softmax(out, V, pi);
+        for (int32_t v = 0; v < V; ++v) { it[v].z = out[v]; it[v].v = v; }
+        qsort(it, (size_t)V, sizeof(warp_item), warp_desc);
+        double above = 0.0;                 /* mass of the tokens strictly more probable than the group */
+        int32_t s = 0;
+        while (s < V && it[s].z > -INFINITY) {
+            int32_t e = s;
+            double group = 0.0;
+            while (e < V && it[e].z == it[s].z) { group += pi[it[e].v]; ++e; }
+            const double gap = fabs(above - top_p);
+            if (gap < *margin_out) *margin_out = gap;
+            if (!(above < top_p))
+                for (int32_t i = s; i < e; ++i) out[it[i].v] = -INFINITY;
+            above += group;
+            s = e;
+        }
+        free(pi);
+    }
+    free(it);
+}
+
 /* ---------------------------------------------------------------- KDE and Bayes (Sec. 4.4) */
 
 /* sample standard deviation (n-1 in the denominator); 0 for n<2 */
@@ -293,7 +372,7 @@ static void position_math(const void* zd, const void* zt, int32_t dtype, int32_t
                           const float* u_target, double* H_d, double* H_t, double* lse_d,
                           double* lse_t, double* jsd, double* dist, int32_t* y,
                           double* y_margin) {
-    size_t esz = dtype == ORACLE_BF16 ? 2 : 4;
+    size_t esz = elt_size(dtype);
 #pragma omp parallel for schedule(dynamic, 1)
     for (int32_t i = 0; i <= K_t; ++i) {
         double* zz = (double*)malloc(sizeof(double) * (size_t)V);
@@ -408,7 +487,7 @@ void oracle_vanilla_round(const void* zd, const void* zt, int32_t dtype, int32_t
                           const int32_t* x, const float* u_accept, double u_resample,
                           double* alpha, int32_t* accept_len, int32_t* next_token,
                           double* resample_margin) {
-    size_t esz = dtype == ORACLE_BF16 ? 2 : 4;
+    size_t esz = elt_size(dtype);
     double* zz = (double*)malloc(sizeof(double) * (size_t)V);
     double* p = (double*)malloc(sizeof(double) * (size_t)V);
     double* q = (double*)malloc(sizeof(double) * (size_t)V);
@@ -485,7 +564,7 @@ int32_t oracle_argmax(const void* z, int32_t dtype, int32_t V) {
 void oracle_greedy_round(const void* zt, int32_t dtype, int32_t V, int64_t t_row_stride, int32_t K,
                          const int32_t* x, int32_t* argmax_out, int32_t* accept_len,
                          int32_t* next_token) {
-    size_t esz = dtype == ORACLE_BF16 ? 2 : 4;
+    size_t esz = elt_size(dtype);
     int32_t w = K;
     for (int32_t i = 0; i <= K; ++i) argmax_out[i] = -2;
     for (int32_t i = 0; i < K; ++i) {

@@ -9,6 +9,9 @@ import os
 from math import exp, log, pi, sqrt
 
 ln2, ln3 = log(2.0), log(3.0)
+dy8 = [1 / 2, 1 / 4, 1 / 8, 1 / 16, 1 / 32, 1 / 64, 1 / 128, 1 / 128]
+s_half = sum(sqrt(x) for x in dy8)
+s_sq = sum(x * x for x in dy8)
 h = 0.2 * 2.25 ** (-0.2)
 norm = 3.0 * h * sqrt(2.0 * pi)
 VALUES = {
@@ -23,6 +26,11 @@ VALUES = {
     "kde_three_point": {"std": 0.2, "h_silverman": h, "h_scott": 0.2 * 3.0 ** (-0.2),
                         "f_0.4": (1.0 + 2.0 * exp(-0.5 * (0.2 / h) ** 2)) / norm,
                         "f_0.2": (1.0 + exp(-0.5 * (0.2 / h) ** 2) + exp(-0.5 * (0.4 / h) ** 2)) / norm},
+    "warp_dyadic_v8": {"t2_p0": sqrt(0.5) / s_half, "t2_p7": sqrt(1 / 128) / s_half,
+                       "thalf_p0": 0.25 / s_sq, "thalf_p1": (1 / 16) / s_sq,
+                       "topk3_H": log(7.0) - (10.0 / 7.0) * ln2, "topk3_lse": log(7.0 / 8.0),
+                       "topp08_margin": 0.05,
+                       "topp074_H": ln3 - (2.0 / 3.0) * ln2, "topp074_lse": log(0.75)},
 }
 
 if __name__ == "__main__":

@@ -616,3 +616,130 @@ def test_gen_only_feedback_is_the_running_mean_of_rejected_entropies():
     assert st.nE.value == 2 and st.T_G.value == 2.25
     oracle.gen_only_update(st, H, 2, 3)                        # accept_len beyond the window: ignored
     assert st.nE.value == 2 and (st.nA.value, st.nR.value) == (0, 0)
+
+
+# ------------------------------------------------------------------ adjusted distribution (Sec. 2.1.1)
+
+def test_warp_identities_leave_the_row_alone():
+    z = rng.normal(size=50) * 3
+    for k, p in [(0, 1.0), (50, 1.0), (77, 1.0), (-1, 1.5)]:
+        out, margin = oracle.warp(z, 1.0, k, p)
+        assert np.array_equal(out, z) and margin == math.inf
+    z32 = z.astype(np.float32)
+    assert np.array_equal(oracle.warp(z32)[0], z32.astype(np.float64))
+    assert np.array_equal(oracle.warp(bf16_bits(z32))[0], oracle.widen(bf16_bits(z32)))
+
+
+def test_warp_golden_dyadic_row(golden):
+    c = golden["warp_dyadic_v8"]
+    e = c["expect"]
+    z = np.log(np.array(c["p"]))
+    p2 = oracle.softmax(oracle.warp(z, 2.0)[0])[0]
+    assert p2[0] == pytest.approx(e["t2_p0"], abs=1e-14) and p2[7] == pytest.approx(e["t2_p7"], abs=1e-14)
+    ph = oracle.softmax(oracle.warp(z, 0.5)[0])[0]
+    assert ph[0] == pytest.approx(e["thalf_p0"], abs=1e-14) and ph[1] == pytest.approx(e["thalf_p1"], abs=1e-14)
+    zk, _ = oracle.warp(z, 1.0, 3, 1.0)
+    assert list(np.isfinite(zk)) == [True] * 3 + [False] * 5
+    pk, lse = oracle.softmax(zk)
+    assert lse == pytest.approx(e["topk3_lse"], abs=1e-14)
+    assert oracle.entropy(pk) == pytest.approx(e["topk3_H"], abs=1e-14)
+    assert pk[:3] == pytest.approx([4 / 7, 2 / 7, 1 / 7], abs=1e-15)
+    zp, margin = oracle.warp(z, 1.0, 0, 0.8)
+    assert np.array_equal(np.isfinite(zp), np.isfinite(zk)) and margin == pytest.approx(e["topp08_margin"], abs=1e-12)
+    zq, _ = oracle.warp(z, 1.0, 0, 0.74)
+    assert list(np.isfinite(zq)) == [True] * 2 + [False] * 6
+    pq, lse = oracle.softmax(zq)
+    assert lse == pytest.approx(e["topp074_lse"], abs=1e-14)
+    assert oracle.entropy(pq) == pytest.approx(e["topp074_H"], abs=1e-14)
+
+
+def test_warp_temperature_is_a_power_of_the_distribution():
+    z = rng.normal(size=300) * 2
+    p, _ = oracle.softmax(z)
+    for T in (0.3, 0.7, 1.9):
+        pT, lseT = oracle.softmax(oracle.warp(z, T)[0])
+        ref = p ** (1.0 / T)
+        assert np.allclose(pT, ref / ref.sum(), rtol=1e-12, atol=0)
+        assert lseT == pytest.approx(np.log(np.exp(z / T - z.max() / T).sum()) + z.max() / T, abs=1e-12)
+
+
+def test_warp_top_k_against_a_partition_and_ties_stay_together():
+    z = rng.normal(size=1000)
+    for k in (1, 2, 17, 999):
+        out, _ = oracle.warp(z, 1.0, k, 1.0)
+        kept = np.flatnonzero(np.isfinite(out))
+        assert set(kept) == set(np.argpartition(-z, k - 1)[:k]) and np.array_equal(out[kept], z[kept])
+    out, _ = oracle.warp(np.array([3.0, 2.0, 2.0, 1.0, 2.0]), 1.0, 2, 1.0)
+    assert list(np.isfinite(out)) == [True, True, True, False, True]          # the tie at rank 2 is not split
+
+
+def test_warp_top_p_against_an_independent_sort_and_is_minimal():
+    """Tie-free rows: the kept set equals the ascending-cumsum rule (drop a token while the
+    mass up to and including it, least probable first, is <= 1 - top_p); its mass reaches
+    top_p and loses that property when its least probable token is removed."""
+    for trial in range(20):
+        z = rng.normal(size=400) * (1 + trial % 4)
+        top_p = float(rng.uniform(0.05, 0.98))
+        out, margin = oracle.warp(z, 1.0, 0, top_p)
+        p, _ = oracle.softmax(z)
+        order = np.argsort(p, kind="stable")
+        csum = np.cumsum(p[order])
+        if margin < 1e-9:
+            continue
+        ref_kept = set(order[csum > 1.0 - top_p])
+        kept = np.flatnonzero(np.isfinite(out))
+        assert set(kept) == ref_kept
+        mass = p[kept].sum()
+        assert mass >= top_p - 1e-12 and mass - p[kept].min() < top_p + 1e-12
+    out, _ = oracle.warp(np.array([0.0, 0.0, 0.0, -1.0]), 1.0, 0, 0.3)
+    assert list(np.isfinite(out)) == [True, True, True, False]                 # ties at the edge stay
+
+
+def test_warp_steps_apply_in_order_temperature_top_k_top_p():
+    z = rng.normal(size=200) * 2
+    a, _ = oracle.warp(z, 0.6, 20, 0.7)
+    b, _ = oracle.warp(oracle.warp(oracle.warp(z, 0.6)[0], 1.0, 20, 1.0)[0], 1.0, 0, 0.7)
+    assert np.array_equal(a, b)
+    c, _ = oracle.warp(oracle.warp(z, 1.0, 0, 0.7)[0], 0.6, 20, 1.0)         # another order: another set
+    assert not np.array_equal(np.isfinite(a), np.isfinite(c))
+
+
+def test_warp_unusable_row_is_scaled_and_not_cut():
+    z = np.array([1.0, np.nan, 3.0, 2.0])
+    out, _ = oracle.warp(z, 2.0, 1, 0.5)
+    assert np.isnan(out[1]) and list(out[[0, 2, 3]]) == [0.5, 1.5, 1.0]
+    out, _ = oracle.warp(np.full(4, -np.inf), 1.0, 2, 0.5)
+    assert np.all(np.isneginf(out))
+
+
+def test_warped_rows_put_mass_on_the_exact_ends_of_the_distance():
+    """Sec. 4.4 observes many distances of exactly 0 or 1; cut supports are where they come
+    from: top-1 rows coincide or are disjoint, wider cuts give distances strictly between."""
+    zd, zt = rng.normal(size=64), rng.normal(size=64)
+    zt[int(np.argmax(zd))] = zt.max() + 1.0                                   # same most probable token
+    p, q = oracle.softmax(oracle.warp(zt, 1.0, 1)[0])[0], oracle.softmax(oracle.warp(zd, 1.0, 1)[0])[0]
+    assert oracle.js_distance_rows(p, q)[0] == 0.0
+    zt2 = zt.copy()
+    zt2[int(np.argmin(zd))] = zt2.max() + 1.0
+    p2 = oracle.softmax(oracle.warp(zt2, 1.0, 1)[0])[0]
+    assert oracle.js_distance_rows(p2, q)[0] == 1.0
+    p5, q5 = oracle.softmax(oracle.warp(zt, 1.0, 5)[0])[0], oracle.softmax(oracle.warp(zd, 1.0, 5)[0])[0]
+    assert 0.0 < oracle.js_distance_rows(p5, q5)[0] < 1.0
+
+
+def test_rounds_accept_warped_float64_rows():
+    """The round functions take the warped rows as they are (float64): a draft step on a
+    top-k row never samples a cut token, and the vanilla accept ratio is 0 for a candidate
+    the target's cut removed."""
+    z = (rng.normal(size=(1, 32)) * 2).astype(np.float32)
+    zk, _ = oracle.warp(z, 0.8, 4, 1.0)
+    for u in np.linspace(0.01, 0.99, 25):
+        d = oracle.draft_step(zk[0], float(u), 0.0)
+        assert np.isfinite(zk[0, d["token"]])
+    zd = rng.normal(size=(1, 32))
+    zt = np.stack([zd[0] + 0.1, rng.normal(size=32)])
+    x = int(np.argmax(zd[0]))
+    ztw = zt.copy()
+    ztw[0, x] = -np.inf
+    ov = oracle.vanilla_round(zd, ztw, [x], [0.5], 0.3)
+    assert ov["alpha"][0] == 0.0 and ov["accept_len"] == 0 and ov["next_token"] != x
