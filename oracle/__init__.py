@@ -76,7 +76,7 @@ def lib():
     L.oracle_greedy_round.restype = None
     L.oracle_gen_only_update.argtypes = [_P, _P, _P, _P, _I, _I]
     L.oracle_gen_only_update.restype = None
-    L.oracle_warp_logits.argtypes = [_P, _I, _D, _I, _D, _P, _P]
+    L.oracle_warp_logits.argtypes = [_P, _I, _D, _I, _D, _D, _P, _P, _P]
     L.oracle_warp_logits.restype = None
     return L
 
@@ -116,19 +116,24 @@ def widen(z: np.ndarray) -> np.ndarray:
     return out
 
 
-def warp(z: np.ndarray, temperature: float = 1.0, top_k: int = 0, top_p: float = 1.0) -> tuple:
+def warp(z: np.ndarray, temperature: float = 1.0, top_k: int = 0, top_p: float = 1.0,
+         band: Optional[float] = None) -> tuple:
     """Adjusted distribution of Sec. 2.1.1 as logits (float64, -inf where a token is cut), for
-    one row or a stack of rows; also the smallest top-p decision margin over the rows."""
+    one row or a stack of rows; also the smallest top-p decision margin over the rows and, if
+    `band` is given, the largest mass any row has within `band` of a top-p decision."""
     zz = widen(z) if z.dtype != np.float64 else np.ascontiguousarray(z)
     V = zz.shape[-1]
     flat = zz.reshape(-1, V)
     out = np.empty_like(flat)
-    margin = math.inf
+    margin, band_mass = math.inf, 0.0
     for r in range(flat.shape[0]):
-        m = _D(0.0)
+        m, bm = _D(0.0), _D(0.0)
         lib().oracle_warp_logits(flat[r].ctypes.data, V, float(temperature), int(top_k), float(top_p),
-                                 out[r].ctypes.data, C.byref(m))
+                                 float(band or 0.0), out[r].ctypes.data, C.byref(m), C.byref(bm))
         margin = min(margin, m.value)
+        band_mass = max(band_mass, bm.value)
+    if band is not None:
+        return out.reshape(zz.shape), margin, band_mass
     return out.reshape(zz.shape), margin
 
 

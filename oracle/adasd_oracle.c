@@ -233,12 +233,15 @@ static int warp_desc(const void* a, const void* b) {
  *
  * margin_out: the smallest |mass of the strictly more probable tokens - top_p| over the
  * groups of equally probable tokens, i.e. how close the top-p decision came to going the
- * other way (+inf when top-p is off).  A row with NaN or without a finite logit is
+ * other way (+inf when top-p is off).  band_mass_out: the mass of the groups whose decision
+ * lies within `band` of going the other way (what a checker that sums the same masses in
+ * lower precision may decide differently).  A row with NaN or without a finite logit is
  * returned scaled and uncut.
  */
 void oracle_warp_logits(const double* z, int32_t V, double temperature, int32_t top_k, double top_p,
-                        double* out, double* margin_out) {
+                        double band, double* out, double* margin_out, double* band_mass_out) {
     *margin_out = INFINITY;
+    *band_mass_out = 0.0;
     int bad = 0, finite = 0;
     for (int32_t v = 0; v < V; ++v) {
         out[v] = z[v] / temperature;
@@ -268,6 +271,7 @@ void oracle_warp_logits(const double* z, int32_t V, double temperature, int32_t 
             while (e < V && it[e].z == it[s].z) { group += pi[it[e].v]; ++e; }
             const double gap = fabs(above - top_p);
             if (gap < *margin_out) *margin_out = gap;
+            if (gap < band) *band_mass_out += group;
             if (!(above < top_p))
                 for (int32_t i = s; i < e; ++i) out[it[i].v] = -INFINITY;
             above += group;

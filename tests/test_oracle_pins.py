@@ -743,3 +743,13 @@ def test_rounds_accept_warped_float64_rows():
     ztw[0, x] = -np.inf
     ov = oracle.vanilla_round(zd, ztw, [x], [0.5], 0.3)
     assert ov["alpha"][0] == 0.0 and ov["accept_len"] == 0 and ov["next_token"] != x
+
+
+def test_warp_band_mass_counts_the_groups_near_the_top_p_decision():
+    z = np.log(np.array([1 / 2, 1 / 4, 1 / 8, 1 / 16, 1 / 32, 1 / 64, 1 / 128, 1 / 128]))
+    # the mass above tokens 0..5 is 0, 1/2, 3/4, 7/8, 15/16, 31/32: top_p = 0.76 is 0.01 from token 2's
+    # decision, 0.115 from token 3's, 0.1775 from token 4's and 0.20875 from token 5's
+    assert oracle.warp(z, 1.0, 0, 0.76, band=0.005)[2] == 0.0
+    assert oracle.warp(z, 1.0, 0, 0.76, band=0.02)[2] == pytest.approx(1 / 8, abs=1e-15)
+    assert oracle.warp(z, 1.0, 0, 0.76, band=0.12)[2] == pytest.approx(1 / 8 + 1 / 16, abs=1e-15)
+    assert oracle.warp(z, 1.0, 0, 0.76, band=0.2)[2] == pytest.approx(1 / 8 + 1 / 16 + 1 / 32, abs=1e-15)
