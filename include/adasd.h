@@ -220,6 +220,34 @@ int adasd_gen_only_update(adasd_ctx* ctx, const float* H_draft_dev, const int32_
                           const int32_t* accept_len_dev, void* stream);
 
 /*
+ * The adjusted distribution tokens are sampled from (Sec. 2.1.1: temperature scaling, top-k
+ * sampling, top-p sampling).  Host-side setting of the context; every later
+ * adasd_draft_entropy, adasd_verify and adasd_vanilla_verify on it works on the adjusted
+ * rows: entropies, log-sum-exps, JS distances, accept ratios and every sampled token are
+ * those of softmax(adjust(z)), for draft and target rows alike.
+ *
+ *   temperature   > 0; logits are divided by it.
+ *   top_k         the k most probable tokens stay, tokens whose logit equals the k-th largest
+ *                 stay with it (ties are never split); <= 0 or >= V: off.
+ *   top_p         in (0, 1]; of what top-k left, a token stays iff the tokens strictly more
+ *                 probable than it hold less than top_p of the mass (the smallest
+ *                 most-probable set whose mass reaches top_p, ties at its edge included);
+ *                 1: off.
+ * Applied in that order.  (1, 0, 1) is the default and changes nothing, bit for bit.
+ * Greedy selection (adasd_greedy_verify, argmax drafting) is unaffected: the most probable
+ * token always stays.  adasd_vanilla_verify_static takes no context and applies none.
+ *
+ * Cost: temperature is a constant in the row passes.  With top-k or top-p on, each call first
+ * finds one cutoff logit per row (row_cutoff_kernel: one more read of the rows), and the row
+ * passes read logits below it as -inf.  Rows without a usable maximum are not cut and are
+ * reported by the row pass (ADASD_STATUS_NAN).
+ * The values are read when a call is issued (or captured in a graph), not when it runs.
+ * Returns ADASD_ERR_SHAPE for a temperature that is not a positive finite number or a top_p
+ * outside (0, 1].
+ */
+int adasd_set_warpers(adasd_ctx* ctx, float temperature, int32_t top_k, float top_p);
+
+/*
  * Vanilla verification for callers that must not allocate device memory.  (The paper has
  * no counterpart: this is a packaging variant of adasd_vanilla_verify, same inputs, same
  * outputs, same arithmetic.)

@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
         "adasd_greedy_verify": [P, P, I64, I64, P, P, P, P, P, P],
         "adasd_gen_only_update": [P, P, P, P, P],
         "adasd_selftest_expired_wait": [P, P, I64, I32, P, P, P, P],
+        "adasd_set_warpers": [P, C.c_float, I32, C.c_float],
         "adasd_get_thresholds": [P, P, P, P, P, P],
         "adasd_state_export": [P, I32, P, C.POINTER(C.c_size_t)],
         "adasd_state_import": [P, I32, P, C.c_size_t],
@@ -157,6 +158,10 @@ def adasd_greedy_verify(ctx, target_logits_dev, t_seq_stride, t_row_stride, draf
 
 def adasd_gen_only_update(ctx, H_draft_dev, draft_len_dev, accept_len_dev, stream) -> int:
     return lib().adasd_gen_only_update(ctx, H_draft_dev, draft_len_dev, accept_len_dev, stream)
+
+
+def adasd_set_warpers(ctx, temperature, top_k, top_p) -> int:
+    return lib().adasd_set_warpers(ctx, temperature, top_k, top_p)
 
 
 def adasd_selftest_expired_wait(ctx, logits_dev, row_stride, row, u_dev, H_out_dev, token_out_dev, stream) -> int:
@@ -292,6 +297,10 @@ class Context:
     def gen_only_update(self, H_draft, accept_len, draft_len=None) -> None:
         self._check(adasd_gen_only_update(self.handle, H_draft.data_ptr(), _ptr(draft_len),
                                           accept_len.data_ptr(), self._stream()), "adasd_gen_only_update")
+
+    def set_warpers(self, temperature: float = 1.0, top_k: int = 0, top_p: float = 1.0) -> None:
+        self._check(adasd_set_warpers(self.handle, float(temperature), int(top_k), float(top_p)),
+                    "adasd_set_warpers")
 
     def get_thresholds(self):
         """(T_G, nE, nA, nR) as new device tensors."""

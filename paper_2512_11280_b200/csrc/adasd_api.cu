@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -36,6 +37,15 @@ struct adasd_ctx {
     bool draft_stream;        // the streaming draft kernel is usable for this V / dtype
     bool lse_stream;          // ... and so is the row log-sum-exp kernel of the vanilla mode
     bool sample_stream;       // ... and its sampling kernel (the vocabulary fits its chunk tables)
+    // adjusted distribution (adasd_set_warpers) and the per-row cutoffs a call works out
+    float temperature;
+    int32_t top_k;
+    float top_p;
+    float* cut_t;             // [B,Kmax+1]
+    float* cut_d;             // [B,Kmax]
+    float* cut_row;           // [B] draft step
+    bool cuts_on() const { return (top_k > 0 && top_k < cfg.V) || top_p < 1.f; }
+    bool warp_on() const { return cuts_on() || temperature != 1.f; }
 };
 
 namespace {
@@ -332,6 +342,45 @@ int fill_verify_params(adasd_ctx* ctx, VerifyParams& p, const void* zd, const vo
     p.tail.bw_rule = ctx->cfg.kde_bandwidth;
     p.tail.reject_rule = ctx->cfg.reject_rule;
     p.tail.update = 0;
+    p.inv_temp = 1.f / ctx->temperature;
+    p.c1 = kLog2e / ctx->temperature;
+    if (ctx->cuts_on()) {
+        p.cut_t = ctx->cut_t;
+        p.cut_d = ctx->cut_d;
+    }
+    return ADASD_OK;
+}
+
+// One cutoff logit per needed row (top-k / top-p of the adjusted distribution).
+int launch_cutoffs(adasd_ctx* ctx, const void* z, long long seq_stride, long long row_stride, int R, int extra,
+                   const int32_t* draft_len, const uint8_t* active, float* cut, cudaStream_t stream) {
+    CutParams c;
+    memset(&c, 0, sizeof(c));
+    c.z = z;
+    c.seq_stride = seq_stride;
+    c.row_stride = row_stride;
+    c.draft_len = draft_len;
+    c.active = active;
+    c.cut = cut;
+    c.status = ctx->st.status;
+    c.B = ctx->cfg.B;
+    c.R = R;
+    c.V = ctx->cfg.V;
+    c.extra = extra;
+    c.c1 = 1.4426950408889634 / (double)ctx->temperature;
+    c.top_k = ctx->top_k;
+    c.top_p = ctx->top_p;
+    const long long rows = (long long)c.B * R;
+    const int grid = (int)std::min<long long>(rows, 2LL * ctx->sm_count);
+    const bool vec = vec_ok(z, ctx->cfg.dtype, {seq_stride, row_stride});
+    if (ctx->cfg.dtype == ADASD_BF16) {
+        if (vec) row_cutoff_kernel<__nv_bfloat16, true><<<grid, kCutThreads, 0, stream>>>(c);
+        else row_cutoff_kernel<__nv_bfloat16, false><<<grid, kCutThreads, 0, stream>>>(c);
+    } else {
+        if (vec) row_cutoff_kernel<float, true><<<grid, kCutThreads, 0, stream>>>(c);
+        else row_cutoff_kernel<float, false><<<grid, kCutThreads, 0, stream>>>(c);
+    }
+    CUDA_TRY(cudaGetLastError());
     return ADASD_OK;
 }
 
@@ -341,7 +390,14 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
     const int cs = pick_cluster(ctx, positions);
     const bool vec = vec_ok(p.zd, ctx->cfg.dtype, {p.d_seq, p.d_row}) &&
                      vec_ok(p.zt, ctx->cfg.dtype, {p.t_seq, p.t_row});
-    if (vec && ctx->fast[MODE].iter > 0) {
+    if (ctx->cuts_on()) {
+        if (int rc = launch_cutoffs(ctx, p.zt, p.t_seq, p.t_row, p.Kmax + 1, 1, p.draft_len, nullptr, ctx->cut_t, stream))
+            return rc;
+        if (int rc = launch_cutoffs(ctx, p.zd, p.d_seq, p.d_row, p.Kmax, 0, p.draft_len, nullptr, ctx->cut_d, stream))
+            return rc;
+    }
+    // the staged kernels work on the rows as they are; an adjusted distribution takes the generic ones
+    if (vec && ctx->fast[MODE].iter > 0 && !ctx->warp_on()) {
         // Vanilla mode with enough rows to fill the GPU: log-sum-exps of all rows in one light
         // streaming pass, the accept test per sequence, then the sampling of one position per
         // sequence.  With fewer rows than CTA slots of the streaming pass: everything in the one
@@ -525,7 +581,13 @@ int adasd_create(adasd_ctx** out, const adasd_config* cfg) {
     ALLOC(t.only_pos, B);
     ALLOC(t.q_items, B);
     ALLOC(t.q_ctl, 4);
+    ALLOC(c->cut_t, B * (K + 1));
+    ALLOC(c->cut_d, B * K);
+    ALLOC(c->cut_row, B);
 #undef ALLOC
+    c->temperature = 1.f;
+    c->top_k = 0;
+    c->top_p = 1.f;
     if (rc == ADASD_OK && cudaMemset(t.q_items, 0xFF, B * sizeof(int32_t)) != cudaSuccess) rc = ADASD_ERR_CUDA;
     if (rc == ADASD_OK) fast_setup(c, prop.sharedMemPerBlockOptin);
     if (rc == ADASD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = ADASD_ERR_CUDA;
@@ -589,6 +651,9 @@ static int draft_entropy_impl(adasd_ctx* ctx, const void* logits_dev, int64_t ro
     p.B = ctx->cfg.B;
     p.V = ctx->cfg.V;
     p.expire_row = expire_row;
+    p.inv_temp = 1.f / ctx->temperature;
+    p.c1 = kLog2e / ctx->temperature;
+    if (ctx->cuts_on()) p.cut = ctx->cut_row;
     const int cs = pick_cluster(ctx, p.B);
     const bool vec = vec_ok(logits_dev, ctx->cfg.dtype, {row_stride});
     if (expire_row >= 0 && !(vec && ctx->draft_stream && expire_row < ctx->cfg.B))
@@ -610,7 +675,11 @@ static int draft_entropy_impl(adasd_ctx* ctx, const void* logits_dev, int64_t ro
         a.V = ctx->cfg.V;
         if (int rc = launch_argmax(ctx, a, st)) return rc;
     }
-    if (vec && ctx->draft_stream) {
+    if (ctx->cuts_on()) {
+        if (int rc = launch_cutoffs(ctx, logits_dev, row_stride, 0, 1, 1, nullptr, active_inout_dev, ctx->cut_row, st))
+            return rc;
+    }
+    if (vec && ctx->draft_stream && (!ctx->warp_on() || expire_row >= 0)) {
         const int P = draft_stream_p(ctx);
         // a grid of at most one CTA per SM runs 16 warps per CTA, a larger one 8 (two CTAs per SM)
         const bool big = (long long)p.B * P <= ctx->sm_count && P * kDWBig <= kDMaxEntries;
@@ -771,6 +840,16 @@ int adasd_gen_only_update(adasd_ctx* ctx, const float* H_draft_dev, const int32_
     return ADASD_OK;
 }
 
+int adasd_set_warpers(adasd_ctx* ctx, float temperature, int32_t top_k, float top_p) {
+    if (!ctx) return ADASD_ERR_NULL;
+    if (!(temperature > 0.f) || !std::isfinite(temperature)) return ADASD_ERR_SHAPE;
+    if (!(top_p > 0.f) || top_p > 1.f) return ADASD_ERR_SHAPE;
+    ctx->temperature = temperature;
+    ctx->top_k = top_k < 0 ? 0 : top_k;
+    ctx->top_p = top_p;
+    return ADASD_OK;
+}
+
 int adasd_get_thresholds(adasd_ctx* ctx, float* T_G_dev, int32_t* nE_dev, int32_t* nA_dev,
                          int32_t* nR_dev, void* stream) {
     if (!ctx) return ADASD_ERR_NULL;
@@ -914,6 +993,8 @@ int adasd_vanilla_verify_static(int32_t B, int32_t V, int32_t Kmax, int32_t dtyp
 
     VerifyParams p;
     memset(&p, 0, sizeof(p));
+    p.inv_temp = 1.f;                        // no context, no adjusted distribution
+    p.c1 = kLog2e;
     p.zd = draft_logits_dev;
     p.zt = target_logits_dev;
     p.d_seq = d_seq_stride;

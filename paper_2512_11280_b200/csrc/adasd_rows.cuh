@@ -6,6 +6,7 @@
 
 #include "adasd_device.cuh"
 #include "adasd_tail.cuh"
+#include "adasd_warp.cuh"
 
 namespace adasd {
 
@@ -46,6 +47,11 @@ struct VerifyParams {
     State st;
     TailConfig tail;
     int32_t B, V, Kmax;
+    // adjusted distribution (Sec. 2.1.1): 1 / temperature and, per row, the logit below which
+    // tokens are cut (null: no cut); the staged kernels fold the temperature into c1 = log2 e / T
+    float inv_temp, c1;
+    const float* cut_t;     // [B,Kmax+1]
+    const float* cut_d;     // [B,Kmax]
 };
 
 struct DraftParams {
@@ -61,6 +67,8 @@ struct DraftParams {
     State st;
     int32_t B, V;
     int32_t expire_row;     // self-test of the bounded waits: the row whose first copy is never asked for (-1: none)
+    float inv_temp, c1;     // adjusted distribution: 1 / temperature, log2 e / temperature
+    const float* cut;       // [B] logit below which a row's tokens are cut (null: no cut)
 };
 
 struct RowShared {
@@ -92,12 +100,13 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(DraftParams p) {
     const int NU = (p.V + N - 1) / N;
     const int u0 = (int)((long long)gw * NU / GW), u1 = (int)((long long)(gw + 1) * NU / GW);
     const T* row = reinterpret_cast<const T*>(p.z) + (long long)b * p.row_stride;
+    const RowWarp wr = {p.inv_temp, p.cut ? p.cut[b] : -INFINITY};
 
     // pass A: max, NaN flag
     float vA[2] = {-INFINITY, 0.f};
     for (int u = u0 + lane; u < u1; u += 32) {
         float x[N];
-        load_unit<T, VEC>(row, u, p.V, x);
+        load_unit_w<T, VEC>(row, u, p.V, x, wr);
 #pragma unroll
         for (int j = 0; j < N; ++j) {
             vA[1] = (x[j] != x[j]) ? 1.f : vA[1];
@@ -113,7 +122,7 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(DraftParams p) {
     float vB[2] = {0.f, 0.f};
     for (int u = u0 + lane; u < u1; u += 32) {
         float x[N];
-        load_unit<T, VEC>(row, u, p.V, x);
+        load_unit_w<T, VEC>(row, u, p.V, x, wr);
 #pragma unroll
         for (int j = 0; j < N; ++j) {
             float t = (fmaxf(x[j], kFloor) - m) * kLog2e;
@@ -143,7 +152,7 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(DraftParams p) {
         if (chosen == gw) {
             int tok = warp_scan_select<N>(u0, u1, p.V, base, target, [&](int u, float(&w)[N]) {
                 float x[N];
-                load_unit<T, VEC>(row, u, p.V, x);
+                load_unit_w<T, VEC>(row, u, p.V, x, wr);
 #pragma unroll
                 for (int j = 0; j < N; ++j) w[j] = ex2((fmaxf(x[j], kFloor) - m) * kLog2e);
             });
@@ -192,13 +201,15 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
     const T* rt = reinterpret_cast<const T*>(p.zt) + (long long)b * p.t_seq + (long long)i * p.t_row;
     const T* rd = bonus ? rt
                         : reinterpret_cast<const T*>(p.zd) + (long long)b * p.d_seq + (long long)i * p.d_row;
+    const RowWarp wt = {p.inv_temp, p.cut_t ? p.cut_t[(size_t)b * (Kmax + 1) + i] : -INFINITY};
+    const RowWarp wd = {p.inv_temp, (p.cut_d && !bonus) ? p.cut_d[(size_t)b * Kmax + i] : -INFINITY};
 
     // pass A: maxima, NaN flag, "rows differ" flag
     float vA[4] = {-INFINITY, -INFINITY, 0.f, 0.f};
     for (int u = u0 + lane; u < u1; u += 32) {
         float xt[N], xd[N];
-        load_unit<T, VEC>(rt, u, p.V, xt);
-        if (!bonus) load_unit<T, VEC>(rd, u, p.V, xd);
+        load_unit_w<T, VEC>(rt, u, p.V, xt, wt);
+        if (!bonus) load_unit_w<T, VEC>(rd, u, p.V, xd, wd);
 #pragma unroll
         for (int j = 0; j < N; ++j) {
             if (bonus) xd[j] = xt[j];
@@ -218,8 +229,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
     float vB[2] = {0.f, 0.f};
     for (int u = u0 + lane; u < u1; u += 32) {
         float xt[N], xd[N];
-        load_unit<T, VEC>(rt, u, p.V, xt);
-        if (!bonus) load_unit<T, VEC>(rd, u, p.V, xd);
+        load_unit_w<T, VEC>(rt, u, p.V, xt, wt);
+        if (!bonus) load_unit_w<T, VEC>(rd, u, p.V, xd, wd);
 #pragma unroll
         for (int j = 0; j < N; ++j) {
             vB[0] += ex2((fmaxf(xt[j], kFloor) - mt) * kLog2e);
@@ -242,8 +253,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
     if (MODE == MODE_VANILLA && !bonus && !bad) {
         const int xi = p.x[(size_t)b * Kmax + i];
         if (xi >= 0 && xi < p.V) {
-            float a = fmaf(fmaxf(to_f32(rt[xi]), kFloor) - mt, kLog2e, -lSt);
-            float q = fmaf(fmaxf(to_f32(rd[xi]), kFloor) - md, kLog2e, -lSd);
+            float a = fmaf(fmaxf(apply_warp(to_f32(rt[xi]), wt), kFloor) - mt, kLog2e, -lSt);
+            float q = fmaf(fmaxf(apply_warp(to_f32(rd[xi]), wd), kFloor) - md, kLog2e, -lSd);
             alpha = fminf(1.f, ex2(a - q));
             if (!(ex2(q) > 0.f)) alpha = 1.f;   // q(x) = 0 cannot have been drafted
         } else {
@@ -263,8 +274,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
     if (MODE == MODE_ADASD || need_resid) {
         for (int u = u0 + lane; u < u1; u += 32) {
             float xt[N], xd[N];
-            load_unit<T, VEC>(rt, u, p.V, xt);
-            if (!bonus) load_unit<T, VEC>(rd, u, p.V, xd);
+            load_unit_w<T, VEC>(rt, u, p.V, xt, wt);
+            if (!bonus) load_unit_w<T, VEC>(rd, u, p.V, xd, wd);
 #pragma unroll
             for (int j = 0; j < N; ++j) {
                 float a = fmaf(fmaxf(xt[j], kFloor) - mt, kLog2e, -lSt);
@@ -321,8 +332,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
                 if (from_resid) {
                     tok = warp_scan_select<N>(u0, u1, p.V, base, target, [&](int u, float(&w)[N]) {
                         float xt[N], xd[N];
-                        load_unit<T, VEC>(rt, u, p.V, xt);
-                        load_unit<T, VEC>(rd, u, p.V, xd);
+                        load_unit_w<T, VEC>(rt, u, p.V, xt, wt);
+                        load_unit_w<T, VEC>(rd, u, p.V, xd, wd);
 #pragma unroll
                         for (int j = 0; j < N; ++j) {
                             float pp = ex2(fmaf(fmaxf(xt[j], kFloor) - mt, kLog2e, -lSt));
@@ -333,7 +344,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(VerifyParams p) {
                 } else {
                     tok = warp_scan_select<N>(u0, u1, p.V, base, target, [&](int u, float(&w)[N]) {
                         float xt[N];
-                        load_unit<T, VEC>(rt, u, p.V, xt);
+                        load_unit_w<T, VEC>(rt, u, p.V, xt, wt);
 #pragma unroll
                         for (int j = 0; j < N; ++j)
                             w[j] = ex2((fmaxf(xt[j], kFloor) - mt) * kLog2e);

@@ -36,6 +36,13 @@ TIE_EPS = 2e-6
 # s log2 s with s close to 2 carries the special-function unit's absolute error of 2^-22, and p, q
 # their own rounding.  d = sqrt(D_JS / ln 2) turns an error e of D_JS into e / (2 d ln 2).
 JSD_RESOLUTION = 2.5e-7
+# The device sums the masses of a top-p decision in 2^-40 fixed point: a group of equally
+# probable tokens whose decision lies within WARP_BAND of going the other way may be cut on one
+# side and kept on the other.  While such groups hold less than WARP_MASS of a row, every
+# compared number stays inside its tolerance (H moves by about m |ln m|); a sequence-round with
+# more is not compared and the device state is set to the oracle's.
+WARP_BAND = 1e-8
+WARP_MASS = 5e-6
 
 
 def dist_tolerance(d: float) -> float:
@@ -62,6 +69,7 @@ class Report:
     dist_beyond_tol: int = 0       # of those: |diff| > TOL, inside what fp32 resolves of D_JS at that distance
     p_acc_checked: int = 0         # P(A|d) comparisons made
     p_acc_beyond_tol: int = 0      # of those: |diff| > TOL, inside the band the steepness of P in d allows
+    warp_near: int = 0             # sequence-rounds left out because a top-p cut was too close to call
     max_err: dict = field(default_factory=dict)
     accept_hist: dict = field(default_factory=dict)
     window_hist: dict = field(default_factory=dict)
@@ -77,7 +85,7 @@ class Report:
                       near_threshold=self.near_threshold, flips=self.flips, near_ties=self.near_ties,
                       tie_flips=self.tie_flips, resyncs=self.resyncs, r6_resyncs=self.r6_resyncs,
                       dist_checked=self.dist_checked, dist_beyond_tol=self.dist_beyond_tol,
-                      p_acc_checked=self.p_acc_checked, p_acc_beyond_tol=self.p_acc_beyond_tol,
+                      p_acc_checked=self.p_acc_checked, p_acc_beyond_tol=self.p_acc_beyond_tol, warp_near=self.warp_near,
                       n_rejections=self.n_rejections)
         return dict({k: int(v) for k, v in counts.items()},
                     max_err={k: float(f"{v:.3e}") for k, v in self.max_err.items()},
@@ -94,7 +102,8 @@ class Lockstep:
     def __init__(self, wl: synth.Workload, follow: Optional[List[int]] = None,
                  cluster_size: int = 0, list_capacity: Optional[int] = None,
                  min_kde_samples: int = 2, device: int = 0, check_lists_every: int = 16,
-                 kde_bandwidth: int = 0, reject_rule: int = 0):
+                 kde_bandwidth: int = 0, reject_rule: int = 0,
+                 warpers: Optional[tuple] = None):
         import torch
         import paper_2512_11280_b200 as adasd
         self.torch, self.adasd, self.wl = torch, adasd, wl
@@ -104,6 +113,12 @@ class Lockstep:
         self.ctx = adasd.Context(wl.B, wl.V, wl.K, dtype=wl.dtype, list_capacity=cap,
                                  min_kde_samples=min_kde_samples, cluster_size=cluster_size,
                                  kde_bandwidth=kde_bandwidth, reject_rule=reject_rule, device=device)
+        # adjusted distribution (temperature, top_k, top_p): set on the context, and applied by
+        # the oracle to the host rows before its own steps
+        if warpers is not None:                 # as the library stores them: temperature and top_p in fp32
+            warpers = (float(np.float32(warpers[0])), int(warpers[1]), float(np.float32(warpers[2])))
+            self.ctx.set_warpers(*warpers)
+        self.warpers = warpers
         self.gs = synth.GpuSynth(wl, str(self.dev))
         tdt = torch.bfloat16 if wl.dtype == synth.BF16 else torch.float32
         B, K, V = wl.B, wl.K, wl.V
@@ -171,6 +186,17 @@ class Lockstep:
         # ---- oracle draft phase for the followed sequences (host rows)
         fb = np.array(self.follow, dtype=np.int32)
         hd, ht = synth.host_round(wl, r, fb)
+        skip = set()              # sequences one of whose rows has too much mass on a top-p decision too close to call
+        if self.warpers is not None:
+            def warp_rows(n):
+                d, _, md = oracle.warp(hd[n], *self.warpers, band=WARP_BAND)
+                t, _, mt = oracle.warp(ht[n], *self.warpers, band=WARP_BAND)
+                return d, t, max(md, mt)
+            w = list(self.pool.map(warp_rows, range(len(self.follow))))
+            hd = np.stack([a[0] for a in w])
+            ht = np.stack([a[1] for a in w])
+            skip = {self.follow[n] for n, a in enumerate(w) if a[2] > WARP_MASS}
+            rep.warp_near += len(skip)
         def draft_phase(n):
             b = self.follow[n]
             st, steps = self.states[b], []
@@ -197,7 +223,7 @@ class Lockstep:
                 H_h = self.Hk[k].cpu().numpy()
                 for b in self.follow:
                     steps = o_draft[b]
-                    if k >= len(steps):
+                    if k >= len(steps) or b in skip:
                         continue
                     o = steps[k]
                     self._close("H_draft", float(H_h[b]), o["H"], ctx=f"b={b} k={k}")
@@ -219,6 +245,11 @@ class Lockstep:
         for b in self.follow:
             steps = o_draft[b]
             K_t = len(steps)
+            if b in skip:                       # the oracle's window and tokens are taken as they are
+                self.draft_len[b] = K_t
+                for k, o in enumerate(steps):
+                    self.x[b, k] = o["token"]
+                continue
             if dl_h[b] != K_t:
                 self._fail(f"window b={b}: gpu {dl_h[b]} oracle {K_t}")
             _bump(rep.window_hist, K_t)
@@ -277,6 +308,9 @@ class Lockstep:
             st = self.states[b]
             K_t = len(o_draft[b])
             LA0, LR0, o, ov = o_verify[n]
+            if b in skip:
+                self._resync(b)
+                continue
             rep.positions += K_t + 1
             _bump(rep.accept_hist, o["accept_len"])
             rep.n_rejections += o["rejected"]

@@ -38,6 +38,7 @@ def test_strerror_and_null_arguments():
     assert lib.adasd_destroy(None) == -1
     assert lib.adasd_status(None, None) == -1
     assert lib.adasd_update_thresholds(None, None, None) == -1
+    assert adasd.adasd_set_warpers(None, 1.0, 0, 1.0) == -1
 
 
 def test_error_codes_of_the_header_have_messages_and_match_the_binding():
