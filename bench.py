@@ -186,6 +186,8 @@ def run_ours(args) -> dict:
                         list_capacity=args.prefill + (args.steps + args.warmup + 64) * K + 64, device=local)
     if args.prefill > 0:
         prefill_lists(ctx, B, args.prefill)
+    if args.warpers:
+        ctx.set_warpers(*args.warpers)
     gs = synth.GpuSynth(wl, str(dev))
 
     # input sets resident in HBM, cycled so that consecutive steps never share data;
@@ -321,6 +323,10 @@ def run_ours(args) -> dict:
                    "value_is": "rows read by adasd_verify / adasd_verify time (mean of the timed launches, max over ranks)",
                    "step_rows_per_s_all_calls": whole_job_rate(world, rows_step, args.steps, ms),
                    "kde_list_prefill": args.prefill,
+                   "warpers": None if not args.warpers else
+                   {"temperature": args.warpers[0], "top_k": args.warpers[1], "top_p": args.warpers[2],
+                    "note": "with top-k / top-p on, every call first finds one cutoff logit per row "
+                            "(row_cutoff_kernel): the times include it, the bytes count the rows once"},
                    "draft_entropy": {"us_per_call": 1e3 * draft_ms, "bytes_per_call": B * row_bytes,
                                      "gbs": B * row_bytes / (draft_ms * 1e-3) / 1e9,
                                      "frac_of_peak": B * row_bytes / (draft_ms * 1e-3) / 1e9 / peak,
@@ -751,6 +757,7 @@ def main():
     ap.add_argument("--workload", default="C4", choices=["C1", "C2", "C3", "C4", "C5"])
     ap.add_argument("--prefill", type=int, default=0,
                     help="entries imported into both KDE lists of every sequence before timing (C3, C4)")
+    ap.add_argument("--warpers", default="", help="C3/C4: temperature,top_k,top_p of the adjusted distribution, e.g. 0.8,50,0.95")
     ap.add_argument("--rounds", type=int, default=0, help="C5: rounds replayed (0 = all 1024)")
     ap.add_argument("--sets", type=int, default=4, help="input sets resident in HBM")
     ap.add_argument("--e2e-steps", type=int, default=6)
@@ -758,6 +765,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.warpers:
+        t, k, p_ = args.warpers.split(",")
+        args.warpers = (float(t), int(k), float(p_))
+        if args.workload not in ("C3", "C4"):
+            ap.error("--warpers applies to the fixed-window workloads C3 and C4")
     out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out is not None:
         print(json.dumps(out))

@@ -37,6 +37,7 @@ struct adasd_ctx {
     bool draft_stream;        // the streaming draft kernel is usable for this V / dtype
     bool lse_stream;          // ... and so is the row log-sum-exp kernel of the vanilla mode
     bool sample_stream;       // ... and its sampling kernel (the vocabulary fits its chunk tables)
+    bool cut_hist;            // the one-pass cutoff kernel got its 128 KB of shared memory
     // adjusted distribution (adasd_set_warpers) and the per-row cutoffs a call works out
     float temperature;
     int32_t top_k;
@@ -239,17 +240,26 @@ void fast_setup(adasd_ctx* c, size_t smem_optin) {
     c->draft_stream = false;
     c->lse_stream = false;
     c->sample_stream = false;
+    c->cut_hist = cudaFuncSetAttribute(row_cutoff_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kHistWords * 4) == cudaSuccess;
+    if (!c->cut_hist) cudaGetLastError();
     const int V = c->cfg.V;
     if (c->cfg.dtype == ADASD_BF16 && (V & 7) == 0 && V >= 8192 &&
         (V >> 3) <= kDMaxP * kDW * kDMaxChunks * kDChunkUnits) {
-        if (cudaFuncSetAttribute(draft_stream_kernel<kDW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(draft_stream_kernel<kDW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kDW * 2 * kDChunkBytes) == cudaSuccess &&
-            cudaFuncSetAttribute(draft_stream_kernel<kDWBig>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaFuncSetAttribute(draft_stream_kernel<kDWBig, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kDWBig * 2 * kDChunkBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(draft_stream_kernel<kDW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kDW * 2 * kDChunkBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(draft_stream_kernel<kDWBig, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kDWBig * 2 * kDChunkBytes) == cudaSuccess)
             c->draft_stream = true;
         else
             cudaGetLastError();
-        if (cudaFuncSetAttribute(row_lse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(row_lse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kLW * 2 * kLChunkBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(row_lse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kLW * 2 * kLChunkBytes) == cudaSuccess)
             c->lse_stream = true;
         else
@@ -278,7 +288,7 @@ int draft_stream_p(const adasd_ctx* c) {
     return P;
 }
 
-template <int ITER, int MODE>
+template <int ITER, int MODE, bool WARPED>
 int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
     const long long positions = (long long)p.B * (p.Kmax + 1);
     const adasd_ctx::Fast& f = c->fast[MODE];
@@ -297,13 +307,22 @@ int fast_launch(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&lc, spec_verify_kernel<ITER, MODE>, p, gq));
+    if (WARPED) {
+        // the instantiation for adjusted distributions: same footprint, its own attribute
+        CUDA_TRY(cudaFuncSetAttribute(spec_verify_kernel<ITER, MODE, WARPED>, cudaFuncAttributeMaxDynamicSharedMemorySize, f.smem));
+    }
+    CUDA_TRY(cudaLaunchKernelEx(&lc, spec_verify_kernel<ITER, MODE, WARPED>, p, gq));
     return ADASD_OK;
 }
 
 template <int MODE>
 int fast_launch_iter(adasd_ctx* c, const VerifyParams& p, cudaStream_t stream) {
-#define CALL(I) fast_launch<I, MODE>(c, p, stream)
+    if (c->warp_on()) {
+#define CALL(I) fast_launch<I, MODE, true>(c, p, stream)
+        ADASD_ITER_SWITCH(c->fast[MODE].iter, CALL, ADASD_ERR_SHAPE)
+#undef CALL
+    }
+#define CALL(I) fast_launch<I, MODE, false>(c, p, stream)
     ADASD_ITER_SWITCH(c->fast[MODE].iter, CALL, ADASD_ERR_SHAPE)
 #undef CALL
 }
@@ -371,8 +390,16 @@ int launch_cutoffs(adasd_ctx* ctx, const void* z, long long seq_stride, long lon
     c.top_k = ctx->top_k;
     c.top_p = ctx->top_p;
     const long long rows = (long long)c.B * R;
-    const int grid = (int)std::min<long long>(rows, 2LL * ctx->sm_count);
     const bool vec = vec_ok(z, ctx->cfg.dtype, {seq_stride, row_stride});
+    if (ctx->cfg.dtype == ADASD_BF16 && vec && ctx->cut_hist) {
+        // one pass per row over a histogram of the 65536 bf16 values; a row it cannot do (a value
+        // that occurs 65536 times or more) is left flagged for the radix kernel
+        const int g1 = (int)std::min<long long>(rows, (long long)ctx->sm_count);
+        row_cutoff_hist_kernel<<<g1, kHistThreads, kHistWords * 4, stream>>>(c);
+        CUDA_TRY(cudaGetLastError());
+        c.only_flagged = 1;
+    }
+    const int grid = (int)std::min<long long>(rows, 2LL * ctx->sm_count);
     if (ctx->cfg.dtype == ADASD_BF16) {
         if (vec) row_cutoff_kernel<__nv_bfloat16, true><<<grid, kCutThreads, 0, stream>>>(c);
         else row_cutoff_kernel<__nv_bfloat16, false><<<grid, kCutThreads, 0, stream>>>(c);
@@ -396,8 +423,7 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
         if (int rc = launch_cutoffs(ctx, p.zd, p.d_seq, p.d_row, p.Kmax, 0, p.draft_len, nullptr, ctx->cut_d, stream))
             return rc;
     }
-    // the staged kernels work on the rows as they are; an adjusted distribution takes the generic ones
-    if (vec && ctx->fast[MODE].iter > 0 && !ctx->warp_on()) {
+    if (vec && ctx->fast[MODE].iter > 0) {
         // Vanilla mode with enough rows to fill the GPU: log-sum-exps of all rows in one light
         // streaming pass, the accept test per sequence, then the sampling of one position per
         // sequence.  With fewer rows than CTA slots of the streaming pass: everything in the one
@@ -419,7 +445,11 @@ int launch_verify(adasd_ctx* ctx, const VerifyParams& p, cudaStream_t stream) {
             lp.B = p.B;
             lp.V = p.V;
             lp.Kmax = p.Kmax;
-            row_lse_kernel<<<2 * ctx->sm_count, kLW * 32, kLW * 2 * kLChunkBytes, stream>>>(lp);
+            lp.c1 = p.c1;
+            lp.cut_t = p.cut_t;
+            lp.cut_d = p.cut_d;
+            if (ctx->warp_on()) row_lse_kernel<true><<<2 * ctx->sm_count, kLW * 32, kLW * 2 * kLChunkBytes, stream>>>(lp);
+            else row_lse_kernel<false><<<2 * ctx->sm_count, kLW * 32, kLW * 2 * kLChunkBytes, stream>>>(lp);
             CUDA_TRY(cudaGetLastError());
             vanilla_accept_kernel<<<(p.B + 3) / 4, 128, 0, stream>>>(p, p.sc.only_pos);     // one warp per sequence
             CUDA_TRY(cudaGetLastError());
@@ -679,7 +709,7 @@ static int draft_entropy_impl(adasd_ctx* ctx, const void* logits_dev, int64_t ro
         if (int rc = launch_cutoffs(ctx, logits_dev, row_stride, 0, 1, 1, nullptr, active_inout_dev, ctx->cut_row, st))
             return rc;
     }
-    if (vec && ctx->draft_stream && (!ctx->warp_on() || expire_row >= 0)) {
+    if (vec && ctx->draft_stream) {
         const int P = draft_stream_p(ctx);
         // a grid of at most one CTA per SM runs 16 warps per CTA, a larger one 8 (two CTAs per SM)
         const bool big = (long long)p.B * P <= ctx->sm_count && P * kDWBig <= kDMaxEntries;
@@ -701,10 +731,13 @@ static int draft_entropy_impl(adasd_ctx* ctx, const void* logits_dev, int64_t ro
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = attr;
         lc.numAttrs = 2;
+        const bool warped = ctx->warp_on();
         if (big) {
-            CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDWBig>, p));
+            if (warped) CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDWBig, true>, p));
+            else CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDWBig, false>, p));
         } else {
-            CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDW>, p));
+            if (warped) CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDW, true>, p));
+            else CUDA_TRY(cudaLaunchKernelEx(&lc, draft_stream_kernel<kDW, false>, p));
         }
         return ADASD_OK;
     }

@@ -80,6 +80,26 @@ __device__ __forceinline__ uint32_t bclamp2(uint32_t a) {             // max(a, 
     asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(0xF149F149u));
     return d;
 }
+// Top-k / top-p cut of the adjusted distribution on a packed pair: a half below the row's cutoff
+// (cut2: the cutoff in both halves) becomes the floor value, i.e. probability 0; a NaN is not
+// below anything and stays.  kNoCut2 (-inf, -inf) cuts nothing.
+constexpr uint32_t kNoCut2 = 0xFF80FF80u;
+__device__ __forceinline__ uint32_t bcut2(uint32_t a, uint32_t cut2) {
+    uint32_t m;
+    asm("set.lt.u32.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(a), "r"(cut2));   // 0xFFFF per half that is below
+    return (a & ~m) | (0xF149F149u & m);
+}
+__device__ __forceinline__ void bcut8(uint4& w, uint32_t cut2) {
+    w.x = bcut2(w.x, cut2);
+    w.y = bcut2(w.y, cut2);
+    w.z = bcut2(w.z, cut2);
+    w.w = bcut2(w.w, cut2);
+}
+// the cutoff of a bf16 row (a bf16 value, or -inf) as a packed pair
+__device__ __forceinline__ uint32_t cut_pair(float cut) {
+    const uint32_t h = __float_as_uint(cut) >> 16;
+    return h | (h << 16);
+}
 __device__ __forceinline__ float2 unpack2(uint32_t w) {
     return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
 }

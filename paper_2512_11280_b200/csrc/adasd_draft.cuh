@@ -35,7 +35,8 @@ struct __align__(16) DraftShared {
 
 // NW warps per CTA: 8 (two CTAs per SM) or 16 (one CTA per SM, for grids that do not fill the
 // SMs twice); P * NW <= kDMaxEntries.
-template <int NW>
+// WARPED: an adjusted distribution is set (Sec. 2.1.1); the ordinary instantiation carries none of its code.
+template <int NW, bool WARPED = false>
 __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kernel(DraftParams p) {
     constexpr int kDW = NW;                    // (shadows the namespace constant: warps of THIS kernel)
     extern __shared__ __align__(128) unsigned char dyn_smem[];
@@ -84,6 +85,9 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
             bulk_g2s(bufs + (size_t)(c & 1) * kDChunkBytes, src + (size_t)c * kDChunkBytes, bytes, bar);
         }
     };
+    // adjusted distribution: t = (z - max) log2 e / T, logits below the row's cutoff count as -inf
+    const float c1 = WARPED ? p.c1 : kLog2e;
+    const uint32_t cut2 = (WARPED && p.cut) ? cut_pair(__ldg(p.cut + b)) : kNoCut2;
     float M = kFloorL;                                   // running shift (log2 domain)
     // the largest logit so far (0 while there is none): t = (z - vM) log2 e is exactly 0 for it,
     // so that a one-hot row gets S = 1, T = 0 and H = 0 exactly
@@ -121,6 +125,10 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
                 if (!(ubase + 32 * i < nwu)) W[i] = make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
                 mx = bmax2(bmax2(mx, W[i].x), bmax2(W[i].y, bmax2(W[i].z, W[i].w)));
             }
+            if (WARPED && cut2 != kNoCut2) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) bcut8(W[i], cut2);
+            }
             // both buffers are in registers or free: fetch the chunk after the next
             __syncwarp();
             issue(c + 2);
@@ -128,9 +136,9 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
             if (mm.x != mm.x || mm.y != mm.y) bad = 1u;
             const float vmax = warp_max_f32(fmaxf(mm.x, mm.y));
             if (vmax == INFINITY) bad = 1u;
-            const float Mc = vmax > ADASD_FLOOR_BF ? vmax * kLog2e : kFloorL;
+            const float Mc = vmax > ADASD_FLOOR_BF ? vmax * c1 : kFloorL;
             if (Mc > M) {                                 // raise the shift, rescale what is summed
-                const float d = M > kFloorL ? (vM - vmax) * kLog2e : kFloorL, f = ex2(d);
+                const float d = M > kFloorL ? (vM - vmax) * c1 : kFloorL, f = ex2(d);
                 T2.x = f * fmaf(d, S2.x, T2.x);
                 T2.y = f * fmaf(d, S2.y, T2.y);
                 S2.x *= f;
@@ -138,7 +146,7 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
                 M = Mc;
                 vM = vmax;
             }
-            const float2 nv2 = make_float2(-vM, -vM), L2 = make_float2(kLog2e, kLog2e);
+            const float2 nv2 = make_float2(-vM, -vM), L2 = make_float2(c1, c1);
             float2 Sc = make_float2(0.f, 0.f);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -259,6 +267,7 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
                     for (int i = 0; i < 8; ++i) {
                         const int u = u0 + 32 * i + lane;
                         Wq[i] = u < u1 ? __ldg(row + u) : make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
+                        if (WARPED) bcut8(Wq[i], cut2);
                     }
                     float run = base;
                     int last_pos = -1;
@@ -271,8 +280,8 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const float2 z = unpack2(bclamp2(qw[j]));
-                                wt[2 * j] = ex2(fmaf(z.x, kLog2e, -Mr));
-                                wt[2 * j + 1] = ex2(fmaf(z.y, kLog2e, -Mr));
+                                wt[2 * j] = ex2(fmaf(z.x, c1, -Mr));
+                                wt[2 * j + 1] = ex2(fmaf(z.y, c1, -Mr));
                             }
                             float ls = 0.f;
 #pragma unroll

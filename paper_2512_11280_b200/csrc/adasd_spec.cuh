@@ -72,7 +72,9 @@ struct __align__(16) PosCtx {
     int32_t pos;                  // index into [B, Kmax+1]; >= total: none
     int32_t kt;                   // window K_t of its sequence
     int32_t bonus;                // 1: the sequence's bonus row (target row only)
-    int32_t pad;
+    uint32_t cut_t;               // adjusted distribution: the target row's cutoff logit as a bf16 pair
+    uint32_t cut_d;               // ... the draft row's (kNoCut2: nothing is cut)
+    int32_t pad[3];
 };
 
 // What a compute warp needs after the exchange: p = 2^t_p * at, q = 2^t_q * ad; and, if it
@@ -211,6 +213,22 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
 struct FinOut {
     float Ht, lse_t, Hd, lse_d, jsd, dist;
 };
+// Top-k / top-p cut of one lane's units of a position buffer, in place (iterations are 512 bytes
+// apart; row_b: offset of the draft row, 0 for a bonus row).  Kept out of line: it runs only when
+// an adjusted distribution is set, and must not cost the ordinary path registers.
+__device__ __noinline__ void cut_buffer(unsigned char* sb, int iters, int row_b, uint32_t c2t, uint32_t c2d) {
+    for (int k = 0; k < iters; ++k) {
+        uint4 T = *reinterpret_cast<const uint4*>(sb + k * 512);
+        bcut8(T, c2t);
+        *reinterpret_cast<uint4*>(sb + k * 512) = T;
+        if (row_b) {
+            uint4 D = *reinterpret_cast<const uint4*>(sb + row_b + k * 512);
+            bcut8(D, c2d);
+            *reinterpret_cast<uint4*>(sb + row_b + k * 512) = D;
+        }
+    }
+}
+
 __device__ __forceinline__ FinOut finalize_math(const RowPart* finc, int CS, float Mt, float Md, double A, float PQ,
                                              uint32_t fl, bool near) {
     const int lane = threadIdx.x & 31;
@@ -391,9 +409,12 @@ __device__ __forceinline__ void verify_tail_warp(const TailConfig& cfg, const Ta
 }
 
 // ------------------------------------------------------------------------------------
-template <int ITER, int MODE>
+// WARPED: an adjusted distribution is set (Sec. 2.1.1); the ordinary instantiation carries none of its code.
+template <int ITER, int MODE, bool WARPED = false>
 __global__ void __launch_bounds__(kSThreads, 1)
 spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
+    const float c1 = WARPED ? p.c1 : kLog2e;                   // log2 e / temperature
+    const float inv_temp = WARPED ? p.inv_temp : 1.f;
     constexpr int KH = ITER < kSHead ? ITER : kSHead;          // head iterations: 2^t values in tensor memory
     constexpr int KR = ITER - KH;                              // tail iterations: 2^t values in registers
     static_assert(KR <= kSRegIter, "too many iterations for the register file");
@@ -474,6 +495,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             if (r.pos < total) {
                 const int b = r.pos / K1, i = r.pos - b * K1;
                 c.bonus = (i == r.kt) ? 1 : 0;
+                c.cut_t = (WARPED && p.cut_t) ? cut_pair(__ldg(p.cut_t + r.pos)) : kNoCut2;
+                c.cut_d = (WARPED && p.cut_d && !c.bonus) ? cut_pair(__ldg(p.cut_d + (size_t)b * Kmax + i)) : kNoCut2;
                 c.src_t = (unsigned long long)(reinterpret_cast<const __nv_bfloat16*>(p.zt) + (long long)b * p.t_seq +
                                                (long long)i * p.t_row + (size_t)cu0 * 8);
                 c.src_d = (unsigned long long)(reinterpret_cast<const __nv_bfloat16*>(p.zd) + (long long)b * p.d_seq +
@@ -626,6 +649,22 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             flags_w = __reduce_or_sync(0xFFFFFFFFu, bad | (a_df ? 2u : 0u)) | (has_t ? 0u : 4u) | (has_d ? 0u : 8u);
         };
 
+        // Adjusted distribution with a top-k / top-p cut: before pass A, the logits below the row's
+        // cutoff are overwritten with the clamp value in the buffer (probability 0), so that every
+        // later pass sees the adjusted rows.  The largest logit always stays, and a NaN is not
+        // below anything, so the maxima and the flags of pass A are those of the rows as given.
+        const bool any_cut = WARPED && (p.cut_t != nullptr);      // the same for every position of the launch
+        auto run_a = [&](bool bonus, int n) {
+            if (any_cut && alive && nwu > 0) {
+                bool ok = mbar_wait_bounded(bar_of(n), (uint32_t)(n >> 1) & 1u);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                // (an expired wait is dealt with by pass A)
+                if (ok) cut_buffer(buf_of(n), full ? ITER : ITER - 1, bonus ? 0 : kRowB, pcx(n).cut_t, pcx(n).cut_d);
+            }
+            if (bonus) pass_a(std::true_type{}, n);
+            else pass_a(std::false_type{}, n);
+        };
+
         // ---- pass B: 2^t of every logit of the share, S = sum 2^t, T = sum 2^t t, max |z_t - z_d| --
         // Head iterations [0, KH) park their values in tensor memory, tail iterations [KH, ITER)
         // keep them in registers.  t = (z - max) log2 e is exactly 0 for the largest logit of the
@@ -641,7 +680,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                 bdz = 0.f;
             }
             const float2 nmt = make_float2(nmt_w, nmt_w), nmd = make_float2(nmd_w, nmd_w);
-            const float2 L2 = make_float2(kLog2e, kLog2e), neg1 = make_float2(-1.f, -1.f);
+            const float2 L2 = make_float2(c1, c1), neg1 = make_float2(-1.f, -1.f);
             const unsigned char* sb = buf_of(n);
 #pragma unroll
             for (int k = K0; k < K1; ++k) {
@@ -704,8 +743,8 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const float dz = warp_max_f32(bdz);
             if (lane == 0) {
                 float4* w = reinterpret_cast<float4*>(&sh.wtab[n & 1][warp]);
-                const float Mt_w = (flags_w & 4u) ? kFloorL : -nmt_w * kLog2e;
-                const float Md_w = (flags_w & 8u) ? kFloorL : -nmd_w * kLog2e;
+                const float Mt_w = (flags_w & 4u) ? kFloorL : -nmt_w * c1;
+                const float Md_w = (flags_w & 8u) ? kFloorL : -nmd_w * c1;
                 w[0] = make_float4(Mt_w, St, Tt, Md_w);
                 w[1] = make_float4(Sd, Td, __uint_as_float(flags_w & 3u), dz);
                 mbar_arrive_cta(reinterpret_cast<uint64_t*>(&sh.entry_bar[n & 1]));
@@ -873,8 +912,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
         int n = 0;                 // sequence number of the current position
         if (pcx(0).pos < total) {
             const bool b0 = pcx(0).bonus != 0;
-            if (b0) pass_a(std::true_type{}, 0);
-            else pass_a(std::false_type{}, 0);
+            run_a(b0, 0);
             b_head(b0, 0);
             b_tail(b0, 0);
             publish(b0, 0);
@@ -892,8 +930,7 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             // while the control warps exchange the totals of position n: maxima and the head of
             // pass B of position n + 1 (its 2^t values go to the other half of tensor memory)
             if (npos < total) {
-                if (nbonus) pass_a(std::true_type{}, n + 1);
-                else pass_a(std::false_type{}, n + 1);
+                run_a(nbonus, n + 1);
                 b_head(nbonus, n + 1);
             }
             wait_cta(&sh.scal_bar[par], ph);
@@ -1016,6 +1053,11 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
                     if (x_ok) {
                         ztx = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.zt)[(long long)b * p.t_seq + (long long)i * p.t_row + xi]);
                         zdx = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.zd)[(long long)b * p.d_seq + (long long)i * p.d_row + xi]);
+                        // a candidate below its row's cutoff has probability 0 there
+                        if (WARPED) {
+                            if (ztx < unpack2(pcn.cut_t).x) ztx = -INFINITY;
+                            if (zdx < unpack2(pcn.cut_d).x) zdx = -INFINITY;
+                        }
                     }
                 }
             }
@@ -1075,15 +1117,15 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
             const uint32_t fl = __reduce_or_sync(0xFFFFFFFFu, __float_as_uint(e1.z));
             const bool bad = (fl & 1u) || !(Mt > kFloorL) || !(Md > kFloorL);
             // AdaSD: the two rows are nearly equal everywhere -> pass C in its well-conditioned form
-            const bool near = (MODE == MODE_ADASD) && !bonus && !bad && (fl & 2u) && warp_max_f32(e1.w) <= kSNearDz;
+            const bool near = (MODE == MODE_ADASD) && !bonus && !bad && (fl & 2u) && warp_max_f32(e1.w) * inv_temp <= kSNearDz;
             float alpha = 0.f;
             bool van_accept = true;
             int act = near ? 5 : 1;               // AdaSD: every row draws y_i ~ p_i
             if (MODE == MODE_VANILLA) {
                 if (!bonus) {
                     if (x_ok) {
-                        const float a = fmaf(fmaxf(ztx, ADASD_FLOOR_BF), kLog2e, -Mt) - lg2(St);
-                        const float q = fmaf(fmaxf(zdx, ADASD_FLOOR_BF), kLog2e, -Md) - lg2(Sd);
+                        const float a = fmaf(fmaxf(ztx, ADASD_FLOOR_BF), c1, -Mt) - lg2(St);
+                        const float q = fmaf(fmaxf(zdx, ADASD_FLOOR_BF), c1, -Md) - lg2(Sd);
                         alpha = fminf(1.f, ex2(a - q));
                         if (!(ex2(q) > 0.f)) alpha = 1.f;   // q(x) = 0 cannot have been drafted
                     }

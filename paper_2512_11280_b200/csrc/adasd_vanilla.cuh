@@ -32,6 +32,9 @@ struct LseParams {
     float* lse_t;                              // [B, Kmax + 1]
     uint32_t* status;
     int32_t B, V, Kmax;
+    float c1;                                  // log2 e / temperature (adjusted distribution)
+    const float* cut_t;                        // nullable [B, Kmax + 1]: logit below which a row's tokens are cut
+    const float* cut_d;                        // nullable [B, Kmax]
 };
 
 struct __align__(16) LseShared {
@@ -45,6 +48,7 @@ struct __align__(16) LseShared {
 // twice.  The 8 warps of a CTA split the row into contiguous shares and stream them through
 // two 4 KB buffers each (1-D bulk copies, bounded waits); a warp's copies run on into its share
 // of the CTA's next row, so the pipeline never drains between rows.
+template <bool WARPED>
 __global__ void __launch_bounds__(kLW * 32, 2) row_lse_kernel(LseParams p) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ LseShared sh;
@@ -106,7 +110,13 @@ __global__ void __launch_bounds__(kLW * 32, 2) row_lse_kernel(LseParams p) {
 
     uint32_t n_done = 0;                          // chunks consumed
     int rows_done = 0;
+    const float c1 = WARPED ? p.c1 : kLog2e;
     for (int r = next_row((int)blockIdx.x); r < total; r = next_row(r + (int)gridDim.x)) {
+        uint32_t cut2 = kNoCut2;
+        if (WARPED && p.cut_t) {
+            const int b = r / R, j = r - b * R;
+            cut2 = cut_pair(j <= K ? __ldg(p.cut_t + (size_t)b * (K + 1) + j) : __ldg(p.cut_d + (size_t)b * K + (j - K - 1)));
+        }
         float M = kFloorL, vM = 0.f;              // running shift (log2 domain) and the logit it belongs to
         float2 S2 = make_float2(0.f, 0.f);
         uint32_t bad = 0u;
@@ -132,19 +142,23 @@ __global__ void __launch_bounds__(kLW * 32, 2) row_lse_kernel(LseParams p) {
             }
             __syncwarp();
             issue_next();                         // the chunk is in registers, its buffer free
+            if (WARPED && cut2 != kNoCut2) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) bcut8(W[i], cut2);
+            }
             const float2 mm = unpack2(mx);
             if (mm.x != mm.x || mm.y != mm.y) bad = 1u;
             const float vmax = warp_max_f32(fmaxf(mm.x, mm.y));
             if (vmax == INFINITY) bad = 1u;
-            const float Mc = vmax > ADASD_FLOOR_BF ? vmax * kLog2e : kFloorL;
+            const float Mc = vmax > ADASD_FLOOR_BF ? vmax * c1 : kFloorL;
             if (Mc > M) {                         // raise the shift, rescale what is summed
-                const float f = ex2(M > kFloorL ? (vM - vmax) * kLog2e : kFloorL);
+                const float f = ex2(M > kFloorL ? (vM - vmax) * c1 : kFloorL);
                 S2.x *= f;
                 S2.y *= f;
                 M = Mc;
                 vM = vmax;
             }
-            const float2 nv2 = make_float2(-vM, -vM), L2 = make_float2(kLog2e, kLog2e);
+            const float2 nv2 = make_float2(-vM, -vM), L2 = make_float2(c1, c1);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint32_t w[4] = {W[i].x, W[i].y, W[i].z, W[i].w};
@@ -208,8 +222,11 @@ __global__ void vanilla_accept_kernel(VerifyParams p, int32_t* only_pos) {
             // scaling so that identical rows give exactly 0, alpha exactly 1
             const __nv_bfloat16* zt = reinterpret_cast<const __nv_bfloat16*>(p.zt) + (long long)b * p.t_seq;
             const __nv_bfloat16* zd = reinterpret_cast<const __nv_bfloat16*>(p.zd) + (long long)b * p.d_seq;
-            const float lp = fmaxf(__bfloat162float(zt[(long long)i * p.t_row + xi]), ADASD_FLOOR_BF) - lt;
-            const float lq = fmaxf(__bfloat162float(zd[(long long)i * p.d_row + xi]), ADASD_FLOOR_BF) - ld;
+            // (logits of the adjusted distribution: scaled by 1 / T, -inf below the row's cutoff)
+            const RowWarp wt = {p.inv_temp, p.cut_t ? p.cut_t[(size_t)b * (K + 1) + i] : -INFINITY};
+            const RowWarp wd = {p.inv_temp, p.cut_d ? p.cut_d[idd] : -INFINITY};
+            const float lp = fmaxf(apply_warp(__bfloat162float(zt[(long long)i * p.t_row + xi]), wt), ADASD_FLOOR_BF) - lt;
+            const float lq = fmaxf(apply_warp(__bfloat162float(zd[(long long)i * p.d_row + xi]), wd), ADASD_FLOOR_BF) - ld;
             alpha = fminf(1.f, ex2(__fmul_rn(__fsub_rn(lp, lq), kLog2e)));
             if (!(ex2(__fmul_rn(lq, kLog2e)) > 0.f)) alpha = 1.f;       // q(x) = 0 cannot have been drafted
         }
@@ -296,16 +313,22 @@ __global__ void __launch_bounds__(kVW * 32, 1) vanilla_sample_kernel(VerifyParam
     __syncwarp();
 
     // weights of one 16-byte unit of both rows: p and max(0, p - q)
-    const float nlt = -lt * kLog2e, nld = -ld * kLog2e;
-    auto weights = [&](const uint4& T, const uint4& D, float (&pv)[8], float (&rv)[8]) {
+    // (adjusted distribution: logits scaled by 1 / T, those below the row's cutoff cut)
+    const float nlt = -lt * kLog2e, nld = -ld * kLog2e, c1 = p.c1;
+    const uint32_t cut2t = p.cut_t ? cut_pair(__ldg(p.cut_t + (size_t)b * K1 + i)) : kNoCut2;
+    const uint32_t cut2d = (p.cut_d && !bonus) ? cut_pair(__ldg(p.cut_d + (size_t)b * K + i)) : kNoCut2;
+    auto weights = [&](const uint4& Tin, const uint4& Din, float (&pv)[8], float (&rv)[8]) {
+        uint4 T = Tin, D = Din;
+        bcut8(T, cut2t);
+        bcut8(D, cut2d);
         const uint32_t tw[4] = {T.x, T.y, T.z, T.w}, dw[4] = {D.x, D.y, D.z, D.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float2 zt2 = unpack2(bclamp2(tw[j])), zd2 = unpack2(bclamp2(dw[j]));
-            pv[2 * j] = ex2(fmaf(zt2.x, kLog2e, nlt));
-            pv[2 * j + 1] = ex2(fmaf(zt2.y, kLog2e, nlt));
-            const float q0 = bonus ? 0.f : ex2(fmaf(zd2.x, kLog2e, nld));
-            const float q1 = bonus ? 0.f : ex2(fmaf(zd2.y, kLog2e, nld));
+            pv[2 * j] = ex2(fmaf(zt2.x, c1, nlt));
+            pv[2 * j + 1] = ex2(fmaf(zt2.y, c1, nlt));
+            const float q0 = bonus ? 0.f : ex2(fmaf(zd2.x, c1, nld));
+            const float q1 = bonus ? 0.f : ex2(fmaf(zd2.y, c1, nld));
             rv[2 * j] = fmaxf(pv[2 * j] - q0, 0.f);
             rv[2 * j + 1] = fmaxf(pv[2 * j + 1] - q1, 0.f);
         }

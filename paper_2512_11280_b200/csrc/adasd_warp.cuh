@@ -60,6 +60,7 @@ struct CutParams {
     double c1;                          // log2 e / temperature
     int32_t top_k;                      // <= 0 or >= V: off
     float top_p;                        // >= 1: off
+    int32_t only_flagged;               // 1: only the rows whose cut entry is NaN (left over by row_cutoff_hist_kernel)
 };
 
 constexpr int kCutThreads = 512;
@@ -126,6 +127,10 @@ __global__ void __launch_bounds__(kCutThreads) row_cutoff_kernel(CutParams p) {
         if (p.draft_len) {
             const int kt = max(0, min(p.draft_len[b], p.R - p.extra));
             if (j >= kt + p.extra) continue;
+        }
+        if (p.only_flagged) {
+            const float c = p.cut[(size_t)b * p.R + j];
+            if (c == c) continue;                            // (the same for every thread of the CTA)
         }
         const T* z = reinterpret_cast<const T*>(p.z) + (long long)b * p.seq_stride + (long long)j * p.row_stride;
 
@@ -242,6 +247,200 @@ __global__ void __launch_bounds__(kCutThreads) row_cutoff_kernel(CutParams p) {
             __syncthreads();
         }
         if (threadIdx.x == 0) p.cut[(size_t)b * p.R + j] = lo_key ? CutKey<T>::value(lo_key) : -INFINITY;
+        __syncthreads();
+    }
+}
+
+// ---- bf16 rows that take 16-byte loads: one pass ---------------------------------------------
+//
+// A bf16 logit has 65536 possible values, so ONE pass over the row can count how often each
+// occurs (a histogram in shared memory, two 16-bit counters to a word), and everything else
+// follows from the counts: the k-th largest value, and - because all tokens of a bin have the same
+// logit - the mass of a bin as count * 2^((value - max) log2 e / T), formed in double precision in a
+// fixed order.  A descending scan of the bins (64 per thread, then a prefix over the threads)
+// finds where the count reaches k and where the mass reaches top_p of what top-k left.
+// A value that occurs 65536 times or more in one row wraps its counter; the total then no longer
+// equals V, the row's entry is left NaN, and row_cutoff_kernel (only_flagged) does that row.
+constexpr int kHistThreads = 1024;
+constexpr int kHistWarps = kHistThreads / 32;
+constexpr int kHistWords = 32768;                  // 65536 counters of 16 bits
+constexpr int kHistPerThread = 65536 / kHistThreads;
+
+struct HistShared {
+    float red[kHistWarps];
+    int flag[kHistWarps];
+    long long wcnt[kHistWarps];
+    double wmass[kHistWarps];
+    long long incl_c[kHistThreads];    // inclusive prefix of the counts over the threads (descending keys)
+    double incl_m[kHistThreads];       // ... of the masses
+    float m;
+    int32_t bad;
+    int32_t owner;                     // first thread whose inclusive prefix reaches the threshold
+    uint32_t key_k, key_p;
+};
+
+__global__ void __launch_bounds__(kHistThreads, 1) row_cutoff_hist_kernel(CutParams p) {
+    using KeyT = CutKey<__nv_bfloat16>;
+    extern __shared__ __align__(16) uint32_t hist[];
+    __shared__ HistShared sh;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
+    const int NU = (p.V + 7) / 8;
+    const int total = p.B * p.R;
+    const bool use_k = p.top_k > 0 && p.top_k < p.V;
+    const bool use_p = p.top_p < 1.f;
+
+    for (int row = blockIdx.x; row < total; row += gridDim.x) {
+        const int b = row / p.R, j = row - b * p.R;
+        if (p.active && p.active[b] == 0) continue;
+        if (p.draft_len) {
+            const int kt = max(0, min(p.draft_len[b], p.R - p.extra));
+            if (j >= kt + p.extra) continue;
+        }
+        const __nv_bfloat16* z =
+            reinterpret_cast<const __nv_bfloat16*>(p.z) + (long long)b * p.seq_stride + (long long)j * p.row_stride;
+
+        for (int i = tid; i < kHistWords / 4; i += kHistThreads)
+            reinterpret_cast<uint4*>(hist)[i] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+
+        // the one pass over the row: counts, largest logit, usability
+        float mx = -INFINITY;
+        int bad = 0;
+        for (int u = tid; u < NU; u += kHistThreads) {
+            float x[8];
+            load_unit<__nv_bfloat16, true>(z, u, p.V, x);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                if (u * 8 + q >= p.V) continue;
+                bad |= (x[q] != x[q]);
+                mx = fmaxf(mx, x[q]);
+                const uint32_t key = KeyT::of(x[q]);
+                atomicAdd(&hist[key >> 1], (key & 1u) ? 0x10000u : 1u);
+            }
+        }
+        mx = warp_max(mx);
+        bad = __any_sync(0xFFFFFFFFu, bad);
+        if (lane == 0) {
+            sh.red[warp] = mx;
+            sh.flag[warp] = bad;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            float m = sh.red[0];
+            int bd = sh.flag[0];
+            for (int w = 1; w < kHistWarps; ++w) {
+                m = fmaxf(m, sh.red[w]);
+                bd |= sh.flag[w];
+            }
+            sh.m = m;
+            sh.bad = bd || !(m > -INFINITY) || m == INFINITY;
+            sh.key_k = 0u;
+            sh.key_p = 0u;
+        }
+        __syncthreads();
+        const float m = sh.m;
+        float* const out = p.cut + (size_t)b * p.R + j;
+        if (sh.bad) {                       // an unusable row is not cut; the row pass reports it
+            if (tid == 0) *out = -INFINITY;
+            __syncthreads();
+            continue;
+        }
+
+        // Thread t owns the keys hi, hi - 1, ..., hi - 63 with hi = 65535 - 64 t: in thread order the
+        // bins run from the largest logit down.
+        const uint32_t hi = 65535u - (uint32_t)tid * kHistPerThread;
+        auto count_of = [&](uint32_t key) -> uint32_t {
+            const uint32_t w = hist[key >> 1];
+            return (key & 1u) ? (w >> 16) : (w & 0xFFFFu);
+        };
+        auto mass_of = [&](uint32_t key, uint32_t c) -> double {
+            return (double)c * exp2((double)(fmaxf(KeyT::value(key), kFloor) - m) * p.c1);
+        };
+        // inclusive prefixes over the threads (thread order = descending keys) into sh.incl_c / incl_m
+        auto block_prefix = [&](long long c, double ms) {
+            long long ci = c;
+            double mi = ms;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long tc = __shfl_up_sync(0xFFFFFFFFu, ci, o);
+                const double tm = __shfl_up_sync(0xFFFFFFFFu, mi, o);
+                if (lane >= o) {
+                    ci += tc;
+                    mi += tm;
+                }
+            }
+            __syncthreads();                // (whatever read the tables before is done)
+            if (lane == 31) {
+                sh.wcnt[warp] = ci;
+                sh.wmass[warp] = mi;
+            }
+            if (tid == 0) sh.owner = kHistThreads;
+            __syncthreads();
+            long long cb = 0;
+            double mb = 0.0;
+            for (int w = 0; w < warp; ++w) {
+                cb += sh.wcnt[w];
+                mb += sh.wmass[w];
+            }
+            sh.incl_c[tid] = cb + ci;
+            sh.incl_m[tid] = mb + mi;
+            __syncthreads();
+        };
+
+        long long lc = 0;
+        for (int q = 0; q < kHistPerThread; ++q) lc += count_of(hi - q);
+        block_prefix(lc, 0.0);
+        if (sh.incl_c[kHistThreads - 1] != (long long)p.V) {     // a counter wrapped: left to the radix kernel
+            if (tid == 0) *out = __int_as_float(0x7FC00000);
+            __syncthreads();
+            continue;
+        }
+        if (use_k) {
+            const long long c_ex = tid ? sh.incl_c[tid - 1] : 0;
+            if (c_ex < p.top_k && sh.incl_c[tid] >= p.top_k) {   // exactly one thread: the counts are integers
+                long long run = c_ex;
+                for (int q = 0; q < kHistPerThread; ++q) {
+                    run += count_of(hi - q);
+                    if (run >= p.top_k) {
+                        sh.key_k = hi - q;
+                        break;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        const uint32_t key_k = sh.key_k;                 // 0: top-k is off
+        uint32_t key_cut = key_k;
+        if (use_p) {
+            // masses of this thread's bins among what top-k left
+            double lm = 0.0;
+            for (int q = 0; q < kHistPerThread; ++q) {
+                const uint32_t key = hi - q, c = count_of(key);
+                if (c && key >= key_k) lm += mass_of(key, c);
+            }
+            block_prefix(0, lm);
+            // top_p of the mass top-k left; the first thread whose prefix reaches it holds the cut
+            const double thr = (double)p.top_p * sh.incl_m[kHistThreads - 1];
+            if (sh.incl_m[tid] >= thr) atomicMin(&sh.owner, tid);
+            __syncthreads();
+            if (tid == sh.owner) {
+                double run = tid ? sh.incl_m[tid - 1] : 0.0;
+                uint32_t found = 0u, last = 0u;
+                for (int q = 0; q < kHistPerThread && !found; ++q) {
+                    const uint32_t key = hi - q, c = count_of(key);
+                    if (!c || key < key_k) continue;
+                    last = key;
+                    run += mass_of(key, c);
+                    if (run >= thr) found = key;
+                }
+                // (rounding between the prefix and the walk: the last bin with mass, or, if this
+                // thread has none, everything below the threads before it)
+                sh.key_p = found ? found : (last ? last : hi);
+            }
+            __syncthreads();
+            key_cut = max(key_k, sh.key_p);
+        }
+        if (tid == 0) *out = key_cut ? KeyT::value(key_cut) : -INFINITY;
         __syncthreads();
     }
 }

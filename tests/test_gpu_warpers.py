@@ -49,6 +49,18 @@ def test_lockstep_rounds_under_warpers(torch, V, dtype, warpers):
     assert len(rep.accept_hist) >= 3, s
 
 
+def test_many_rows_take_the_three_kernel_vanilla_path_under_warpers(torch):
+    """352 rows a round: adasd_vanilla_verify runs row_lse_kernel, vanilla_accept_kernel and
+    vanilla_sample_kernel, adasd_verify the warp-specialised kernel, all on the adjusted rows."""
+    from tests.lockstep import Lockstep
+    wl = synth.WORKLOADS["C3"].scaled(name="warp_manyrows", B=32, K=5, V=8200, rounds=8)
+    rep = Lockstep(wl, follow=[0, 7, 13, 21, 30, 31], min_kde_samples=3, check_lists_every=4,
+                   warpers=(0.8, 50, 0.95)).run()
+    s = rep.summary()
+    assert s["flips"] <= s["near_threshold"] + s["tie_flips"] and s["warp_near"] <= 2, s
+    assert len(rep.vanilla_accept_hist) >= 3, s
+
+
 def test_adaptive_windows_under_warpers(torch):
     from tests.lockstep import Lockstep
     wl = synth.WORKLOADS["C5"].scaled(name="warp_adaptive", B=6, K=8, V=8200, rounds=40)
@@ -132,3 +144,35 @@ def test_identity_settings_change_nothing_and_bad_settings_are_refused(torch, ad
         assert adasd.adasd_set_warpers(ctx.handle, *bad) == adasd.ERR_SHAPE, bad
     assert adasd.adasd_set_warpers(ctx.handle, 1.0, -5, 1.0) == 0          # a negative k is "off"
     assert adasd.adasd_set_warpers(None, 1.0, 0, 1.0) == adasd.ERR_NULL
+
+
+@pytest.mark.parametrize("warpers", [(1.0, 50, 1.0), (0.9, 0, 0.9), (1.1, 300, 0.97)])
+def test_a_value_that_fills_most_of_a_row_does_not_break_the_cut(torch, adasd, warpers):
+    """100000 tokens: one logit value taken by more than 65536 of them (the one-pass kernel counts
+    occurrences in 16 bits and must hand such a row over), a row that is one value throughout, and
+    ordinary rows in between; entropy, log-sum-exp and the sampled token against the oracle."""
+    B, V = 5, 100000
+    rng = np.random.default_rng(11)
+    z = rng.normal(size=(B, V)).astype(np.float32) * 2.0
+    z[1, :] = -3.0
+    z[1, rng.choice(V, 400, replace=False)] = rng.normal(size=400).astype(np.float32) * 2.0 + 1.0
+    z[3, :] = 0.5
+    zt = torch.tensor(z, device="cuda").to(torch.bfloat16)
+    zh = raw(zt, torch)
+    ctx = adasd.Context(B, V, 1, list_capacity=8)
+    ctx.set_warpers(*warpers)
+    ws = (float(np.float32(warpers[0])), warpers[1], float(np.float32(warpers[2])))
+    u = torch.tensor([0.05, 0.35, 0.55, 0.75, 0.95], device="cuda")
+    H = torch.zeros(B, device="cuda")
+    lse = torch.zeros(B, device="cuda")
+    tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+    for _ in range(2):
+        ctx.draft_entropy(zt, H, u=u, token_out=tok, lse_out=lse)
+    torch.cuda.synchronize()
+    for b in range(B):
+        zw, _, band = oracle.warp(zh[b], *ws, band=1e-8)
+        assert band < 1e-6, "pick another seed: a top-p decision of this row is too close to call"
+        o = oracle.draft_step(zw, float(u[b]), 0.0)
+        assert abs(float(H[b]) - o["H"]) < TOL and abs(float(lse[b]) - o["lse"]) < TOL, (b, float(H[b]), o)
+        assert int(tok[b]) == o["token"] or o["margin"] < 2e-6, (b, int(tok[b]), o)
+    assert ctx.status() == 0
