@@ -256,15 +256,35 @@ __global__ void __launch_bounds__(kCutThreads) row_cutoff_kernel(CutParams p) {
 // A bf16 logit has 65536 possible values, so ONE pass over the row can count how often each
 // occurs (a histogram in shared memory, two 16-bit counters to a word), and everything else
 // follows from the counts: the k-th largest value, and - because all tokens of a bin have the same
-// logit - the mass of a bin as count * 2^((value - max) log2 e / T), formed in double precision in a
-// fixed order.  A descending scan of the bins (64 per thread, then a prefix over the threads)
-// finds where the count reaches k and where the mass reaches top_p of what top-k left.
+// logit - the mass of a bin as count * 2^((value - max) log2 e / T).  A descending scan of the bins
+// (64 per thread, then a prefix over the threads, in double precision and a fixed order) finds
+// where the count reaches k and where the mass reaches top_p of what top-k left.
 // A value that occurs 65536 times or more in one row wraps its counter; the total then no longer
 // equals V, the row's entry is left NaN, and row_cutoff_kernel (only_flagged) does that row.
+// The pass works on the packed bf16 pairs as they are loaded (the order-preserving key of a value
+// is three integer operations on its 16 bits): the integer pipe is what bounds it.
 constexpr int kHistThreads = 1024;
 constexpr int kHistWarps = kHistThreads / 32;
 constexpr int kHistWords = 32768;                  // 65536 counters of 16 bits
 constexpr int kHistPerThread = 65536 / kHistThreads;
+static_assert(kHistPerThread == 64, "a thread's keys share bits 6..15");
+
+// Order-preserving key of a bf16 bit pattern (-0 and +0 get neighbouring keys; a cut between them
+// keeps both, because the row passes compare values).
+__device__ __forceinline__ uint32_t hist_key(uint32_t h) { return h ^ (((h >> 15) * 0x7FFFu) + 0x8000u); }
+// Word of the histogram that holds a key's counter.  Two keys 32768 apart share a word (neighbouring
+// values, which are busy together, do not); the low five bits are mixed with bits 6..10 so that the
+// scan, in which the threads of a warp read keys 64 apart, finds them in 32 different banks.
+__device__ __forceinline__ uint32_t hist_slot(uint32_t key) { return (key & 0x7FFFu) ^ ((key >> 6) & 31u); }
+__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t h) {
+    const uint32_t key = hist_key(h);
+    atomicAdd(&hist[hist_slot(key)], 1u + (key >> 15) * 0xFFFFu);      // low or high half of the word
+}
+__device__ __forceinline__ uint32_t cut_bmax2(uint32_t a, uint32_t b) {   // NaN-propagating bf16x2 max
+    uint32_t d;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 
 struct HistShared {
     float red[kHistWarps];
@@ -284,7 +304,7 @@ __global__ void __launch_bounds__(kHistThreads, 1) row_cutoff_hist_kernel(CutPar
     extern __shared__ __align__(16) uint32_t hist[];
     __shared__ HistShared sh;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
-    const int NU = (p.V + 7) / 8;
+    const int NUF = p.V >> 3;                  // full 16-byte units of a row
     const int total = p.B * p.R;
     const bool use_k = p.top_k > 0 && p.top_k < p.V;
     const bool use_p = p.top_p < 1.f;
@@ -296,6 +316,7 @@ __global__ void __launch_bounds__(kHistThreads, 1) row_cutoff_hist_kernel(CutPar
             const int kt = max(0, min(p.draft_len[b], p.R - p.extra));
             if (j >= kt + p.extra) continue;
         }
+        float* const out = p.cut + (size_t)b * p.R + j;
         const __nv_bfloat16* z =
             reinterpret_cast<const __nv_bfloat16*>(p.z) + (long long)b * p.seq_stride + (long long)j * p.row_stride;
 
@@ -303,22 +324,38 @@ __global__ void __launch_bounds__(kHistThreads, 1) row_cutoff_hist_kernel(CutPar
             reinterpret_cast<uint4*>(hist)[i] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
 
-        // the one pass over the row: counts, largest logit, usability
-        float mx = -INFINITY;
-        int bad = 0;
-        for (int u = tid; u < NU; u += kHistThreads) {
-            float x[8];
-            load_unit<__nv_bfloat16, true>(z, u, p.V, x);
+        // the pass over the row: counts, largest logit, usability.  Four units of a thread are asked
+        // for before the first is used: a CTA alone on its SM has to keep enough loads in flight.
+        uint32_t mxp = 0xFF80FF80u;            // (-inf, -inf)
+        {
+            const uint4* zq = reinterpret_cast<const uint4*>(z);
+            for (int u0 = tid; u0 < NUF; u0 += 4 * kHistThreads) {
+                uint4 r[4];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                if (u * 8 + q >= p.V) continue;
-                bad |= (x[q] != x[q]);
-                mx = fmaxf(mx, x[q]);
-                const uint32_t key = KeyT::of(x[q]);
-                atomicAdd(&hist[key >> 1], (key & 1u) ? 0x10000u : 1u);
+                for (int i = 0; i < 4; ++i) r[i] = __ldg(zq + min(u0 + i * kHistThreads, NUF - 1));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (u0 + i * kHistThreads < NUF) {
+                        const uint32_t w[4] = {r[i].x, r[i].y, r[i].z, r[i].w};
+                        mxp = cut_bmax2(cut_bmax2(mxp, cut_bmax2(w[0], w[1])), cut_bmax2(w[2], w[3]));
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            hist_add(hist, w[q] & 0xFFFFu);
+                            hist_add(hist, w[q] >> 16);
+                        }
+                    }
+                }
             }
+            if (tid == 0)                       // the ragged end of a row whose length is no multiple of 8
+                for (int v = NUF * 8; v < p.V; ++v) {
+                    const uint32_t h = (uint32_t)__bfloat16_as_ushort(z[v]);
+                    mxp = cut_bmax2(mxp, h | (h << 16));
+                    hist_add(hist, h);
+                }
         }
-        mx = warp_max(mx);
+        const float m0 = __uint_as_float(mxp << 16), m1 = __uint_as_float(mxp & 0xFFFF0000u);
+        int bad = (m0 != m0) || (m1 != m1);
+        float mx = warp_max(fmaxf(m0, m1));
         bad = __any_sync(0xFFFFFFFFu, bad);
         if (lane == 0) {
             sh.red[warp] = mx;
@@ -339,7 +376,6 @@ __global__ void __launch_bounds__(kHistThreads, 1) row_cutoff_hist_kernel(CutPar
         }
         __syncthreads();
         const float m = sh.m;
-        float* const out = p.cut + (size_t)b * p.R + j;
         if (sh.bad) {                       // an unusable row is not cut; the row pass reports it
             if (tid == 0) *out = -INFINITY;
             __syncthreads();
@@ -347,14 +383,21 @@ __global__ void __launch_bounds__(kHistThreads, 1) row_cutoff_hist_kernel(CutPar
         }
 
         // Thread t owns the keys hi, hi - 1, ..., hi - 63 with hi = 65535 - 64 t: in thread order the
-        // bins run from the largest logit down.
+        // bins run from the largest logit down.  Its keys share bits 6..15, so their counters sit in
+        // one half of 64 words that differ in a fixed mix of the low five bits.
         const uint32_t hi = 65535u - (uint32_t)tid * kHistPerThread;
+        const uint32_t mix = (hi >> 6) & 31u, half_shift = (hi >> 15) * 16u;
         auto count_of = [&](uint32_t key) -> uint32_t {
-            const uint32_t w = hist[key >> 1];
-            return (key & 1u) ? (w >> 16) : (w & 0xFFFFu);
+            return (hist[(key & 0x7FFFu) ^ mix] >> half_shift) & 0xFFFFu;
         };
+        // count * 2^((value - max) log2 e / T): the exponent in double, its integer part applied as a
+        // power of two, 2^fraction from the special-function unit (to about 1e-7 of the bin's mass)
         auto mass_of = [&](uint32_t key, uint32_t c) -> double {
-            return (double)c * exp2((double)(fmaxf(KeyT::value(key), kFloor) - m) * p.c1);
+            const double t = (double)(fmaxf(KeyT::value(key), kFloor) - m) * p.c1;
+            if (t < -1000.0) return 0.0;
+            const double ti = floor(t);
+            const double w = (double)ex2((float)(t - ti));
+            return (double)c * __longlong_as_double((long long)(1023 + (int)ti) << 52) * w;
         };
         // inclusive prefixes over the threads (thread order = descending keys) into sh.incl_c / incl_m
         auto block_prefix = [&](long long c, double ms) {
@@ -414,10 +457,11 @@ __global__ void __launch_bounds__(kHistThreads, 1) row_cutoff_hist_kernel(CutPar
         if (use_p) {
             // masses of this thread's bins among what top-k left
             double lm = 0.0;
-            for (int q = 0; q < kHistPerThread; ++q) {
-                const uint32_t key = hi - q, c = count_of(key);
-                if (c && key >= key_k) lm += mass_of(key, c);
-            }
+            if (lc && hi >= key_k)
+                for (int q = 0; q < kHistPerThread; ++q) {
+                    const uint32_t key = hi - q, c = count_of(key);
+                    if (c && key >= key_k) lm += mass_of(key, c);
+                }
             block_prefix(0, lm);
             // top_p of the mass top-k left; the first thread whose prefix reaches it holds the cut
             const double thr = (double)p.top_p * sh.incl_m[kHistThreads - 1];

@@ -36,12 +36,13 @@ TIE_EPS = 2e-6
 # s log2 s with s close to 2 carries the special-function unit's absolute error of 2^-22, and p, q
 # their own rounding.  d = sqrt(D_JS / ln 2) turns an error e of D_JS into e / (2 d ln 2).
 JSD_RESOLUTION = 2.5e-7
-# The device sums the masses of a top-p decision in 2^-40 fixed point: a group of equally
+# The device sums the masses of a top-p decision in double precision, except for bf16 rows, where
+# the tokens far below the largest logit are added up from fp32 exponentials: a group of equally
 # probable tokens whose decision lies within WARP_BAND of going the other way may be cut on one
 # side and kept on the other.  While such groups hold less than WARP_MASS of a row, every
 # compared number stays inside its tolerance (H moves by about m |ln m|); a sequence-round with
 # more is not compared and the device state is set to the oracle's.
-WARP_BAND = 1e-8
+WARP_BAND = {synth.BF16: 5e-7, synth.FP32: 1e-8}
 WARP_MASS = 5e-6
 
 
@@ -189,8 +190,8 @@ class Lockstep:
         skip = set()              # sequences one of whose rows has too much mass on a top-p decision too close to call
         if self.warpers is not None:
             def warp_rows(n):
-                d, _, md = oracle.warp(hd[n], *self.warpers, band=WARP_BAND)
-                t, _, mt = oracle.warp(ht[n], *self.warpers, band=WARP_BAND)
+                d, _, md = oracle.warp(hd[n], *self.warpers, band=WARP_BAND[wl.dtype])
+                t, _, mt = oracle.warp(ht[n], *self.warpers, band=WARP_BAND[wl.dtype])
                 return d, t, max(md, mt)
             w = list(self.pool.map(warp_rows, range(len(self.follow))))
             hd = np.stack([a[0] for a in w])

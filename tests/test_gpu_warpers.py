@@ -170,7 +170,7 @@ def test_a_value_that_fills_most_of_a_row_does_not_break_the_cut(torch, adasd, w
         ctx.draft_entropy(zt, H, u=u, token_out=tok, lse_out=lse)
     torch.cuda.synchronize()
     for b in range(B):
-        zw, _, band = oracle.warp(zh[b], *ws, band=1e-8)
+        zw, _, band = oracle.warp(zh[b], *ws, band=5e-7)
         assert band < 1e-6, "pick another seed: a top-p decision of this row is too close to call"
         o = oracle.draft_step(zw, float(u[b]), 0.0)
         assert abs(float(H[b]) - o["H"]) < TOL and abs(float(lse[b]) - o["lse"]) < TOL, (b, float(H[b]), o)
