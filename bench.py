@@ -125,6 +125,14 @@ def sfu_figures(B: int, K: int, V: int, verify_ms: float, clocks) -> dict:
             "frac": achieved / peak, "ops_per_launch": ops}
 
 
+def cuts_on(args, wl) -> bool:
+    """A top-k or top-p cut is set (temperature alone adds no launch)."""
+    if not args.warpers:
+        return False
+    _, k, p = args.warpers
+    return (0 < k < wl.V) or p < 1.0
+
+
 def vanilla_launches(wl, sm_count: int) -> int:
     """Kernels one adasd_vanilla_verify call launches: with enough bf16 rows to fill the GPU
     it runs three (log-sum-exps of all rows, accept test, sampling of one
@@ -336,7 +344,10 @@ def run_ours(args) -> dict:
                 "what": "pinned host logits -> device, adasd_verify through the C ABI, results -> host",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": h_out.numel() * 4,
                 "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": args.steps * (K + 1 + vanilla_launches(wl, torch.cuda.get_device_properties(dev).multi_processor_count)),
+        # with a top-k / top-p cut every draft call adds two launches (the one-pass cutoff kernel and the
+        # radix kernel for the rows it hands over), verify and vanilla verify four each (target and draft rows)
+        "gpu_launches": args.steps * (K + 1 + vanilla_launches(wl, torch.cuda.get_device_properties(dev).multi_processor_count)
+                                      + (2 * K + 8 if cuts_on(args, wl) else 0)),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "adasd_verify", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
