@@ -51,6 +51,15 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
     // window lengths) is touched before this wait, which returns once that kernel is complete.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const bool active = !(p.active && p.active[b] == 0);      // same in every CTA of the cluster
+    // what the last step of the row needs from global memory is asked for now, by the warp that
+    // will need it, so that it is there after the stream: the uniform and the threshold
+    float u_row = 0.f, tg_row = 0.f;
+    int32_t len_row = 0;
+    if (active && rank == 0 && warp == 0) {
+        if (p.u != nullptr) u_row = __ldg(p.u + b);
+        tg_row = p.st.T_G[b];
+        if (p.draft_len) len_row = p.draft_len[b];          // (only this row's CTA ever writes it)
+    }
 
     // this warp's share of the row, in 16-byte units
     const int NU = p.V >> 3;
@@ -208,7 +217,7 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
         int tok = -1;
         const bool sampling = (p.u != nullptr && p.token_out != nullptr);
         if (sampling && !rowbad) {
-            float target = __ldg(p.u + b) * S;
+            float target = u_row * S;
             const float w0 = f0 * e0.y, w1 = f1 * e1.y;
             float i0 = w0, i1 = w1;
 #pragma unroll
@@ -262,51 +271,50 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
                     // the chunk again (4 KB, from L2), all of it in flight at once
                     const uint4* row = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.z) +
                                                                       (long long)b * p.row_stride);
+                    // Lane l takes the units u0 + 8 l .. u0 + 8 l + 7, so that index order is lane order: one
+                    // prefix over the lanes' sums places the crossing in a lane, which walks its 64 tokens.
                     uint4 Wq[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const int u = u0 + 32 * i + lane;
+                        const int u = u0 + lane * 8 + i;
                         Wq[i] = u < u1 ? __ldg(row + u) : make_uint4(0xF149F149u, 0xF149F149u, 0xF149F149u, 0xF149F149u);
                         if (WARPED) bcut8(Wq[i], cut2);
                     }
-                    float run = base;
-                    int last_pos = -1;
+                    float wt[8][8];
+                    float ls = 0.f;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        if (tok < 0 && u0 + 32 * i < u1) {          // same for the whole warp
-                            const int u = u0 + 32 * i + lane;
-                            const uint32_t qw[4] = {Wq[i].x, Wq[i].y, Wq[i].z, Wq[i].w};
-                            float wt[8];
+                        const uint32_t qw[4] = {Wq[i].x, Wq[i].y, Wq[i].z, Wq[i].w};
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float2 z = unpack2(bclamp2(qw[j]));
-                                wt[2 * j] = ex2(fmaf(z.x, c1, -Mr));
-                                wt[2 * j + 1] = ex2(fmaf(z.y, c1, -Mr));
-                            }
-                            float ls = 0.f;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) ls += wt[j];
-                            float li = ls;
-#pragma unroll
-                            for (int o = 1; o < 32; o <<= 1) {
-                                const float t = __shfl_up_sync(0xFFFFFFFFu, li, o);
-                                if (lane >= o) li += t;
-                            }
-                            float cc = run + (li - ls);
-                            int hit = -1;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                cc += wt[j];
-                                if (wt[j] > 0.f) {
-                                    last_pos = u * 8 + j;
-                                    if (hit < 0 && cc > target) hit = u * 8 + j;
-                                }
-                            }
-                            const unsigned mh = __ballot_sync(0xFFFFFFFFu, hit >= 0);
-                            if (mh) tok = __shfl_sync(0xFFFFFFFFu, hit, __ffs(mh) - 1);
-                            run += __shfl_sync(0xFFFFFFFFu, li, 31);
+                        for (int j = 0; j < 4; ++j) {
+                            const float2 z = unpack2(bclamp2(qw[j]));
+                            wt[i][2 * j] = ex2(fmaf(z.x, c1, -Mr));
+                            wt[i][2 * j + 1] = ex2(fmaf(z.y, c1, -Mr));
+                            ls += wt[i][2 * j] + wt[i][2 * j + 1];
                         }
                     }
+                    float li = ls;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const float t = __shfl_up_sync(0xFFFFFFFFu, li, o);
+                        if (lane >= o) li += t;
+                    }
+                    float cc = base + (li - ls);
+                    int hit = -1, last_pos = -1;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            cc += wt[i][j];
+                            if (wt[i][j] > 0.f) {
+                                const int idx = (u0 + lane * 8 + i) * 8 + j;
+                                last_pos = idx;
+                                if (hit < 0 && cc > target) hit = idx;
+                            }
+                        }
+                    }
+                    const unsigned mh = __ballot_sync(0xFFFFFFFFu, hit >= 0);
+                    if (mh) tok = __shfl_sync(0xFFFFFFFFu, hit, __ffs(mh) - 1);
                     if (tok < 0) {
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xFFFFFFFFu, last_pos, o));
@@ -320,9 +328,9 @@ __global__ void __launch_bounds__(NW * 32, NW == kDW ? 2 : 1) draft_stream_kerne
             p.H_out[b] = H;
             if (p.lse_out) p.lse_out[b] = lse;
             if (sampling) p.token_out[b] = tok;
-            const bool stop = H > p.st.T_G[b];   // strict; NaN never stops
+            const bool stop = H > tg_row;   // strict; NaN never stops
             if (p.stop_out) p.stop_out[b] = stop ? 1 : 0;
-            if (p.draft_len) p.draft_len[b] += 1;
+            if (p.draft_len) p.draft_len[b] = len_row + 1;
             if (p.active && stop) p.active[b] = 0;
         }
     }
