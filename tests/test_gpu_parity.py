@@ -482,8 +482,10 @@ def test_repeatable_bitwise(torch, adasd):
 
 # ------------------------------------------------------------------ CUDA graph replay
 
-def test_adaptive_round_in_a_cuda_graph_replays_like_eager_calls(torch, adasd):
-    """One whole adaptive round (inputs of the round the device counter names, draft steps
+@pytest.mark.parametrize("warpers", [None, (0.8, 40, 0.95)])
+def test_adaptive_round_in_a_cuda_graph_replays_like_eager_calls(torch, adasd, warpers):
+    """(With and without an adjusted distribution: its cutoff kernels are launches like the others.)
+    One whole adaptive round (inputs of the round the device counter names, draft steps
     with the stop check, verification with the fused threshold update) is captured ONCE in a
     CUDA graph; replaying it R times must leave the sequences in exactly the state that the
     same R rounds issued call by call leave them in: the hot calls launch from device-resident
@@ -496,6 +498,8 @@ def test_adaptive_round_in_a_cuda_graph_replays_like_eager_calls(torch, adasd):
 
     def build():
         ctx = adasd.Context(B, V, K, dtype=wl.dtype, list_capacity=256, device=0)
+        if warpers:
+            ctx.set_warpers(*warpers)
         gs = synth.GpuSynth(wl, str(dev))
         f32, i32 = dict(dtype=torch.float32, device=dev), dict(dtype=torch.int32, device=dev)
         zd = torch.empty((B, K, V), dtype=torch.bfloat16, device=dev)
