@@ -176,3 +176,40 @@ def test_a_value_that_fills_most_of_a_row_does_not_break_the_cut(torch, adasd, w
         assert abs(float(H[b]) - o["H"]) < TOL and abs(float(lse[b]) - o["lse"]) < TOL, (b, float(H[b]), o)
         assert int(tok[b]) == o["token"] or o["margin"] < 2e-6, (b, int(tok[b]), o)
     assert ctx.status() == 0
+
+
+@pytest.mark.parametrize("V,dtype", [(40000, synth.BF16), (4099, synth.BF16), (3000, synth.FP32)])
+def test_unusable_and_sparse_rows_under_a_cut(torch, adasd, V, dtype):
+    """Rows the cut has to leave alone or nearly so: a row with a NaN (not cut; reported as
+    unusable by the row pass), a row with fewer finite logits than top_k (everything finite
+    stays), a row whose finite logits are all equal, next to an ordinary row."""
+    B = 4
+    rng = np.random.default_rng(5)
+    z = (rng.normal(size=(B, V)) * 2.0).astype(np.float32)
+    z[0, 17] = np.nan
+    z[1, :] = -np.inf
+    z[1, rng.choice(V, 10, replace=False)] = rng.normal(size=10).astype(np.float32)
+    z[2, :] = -np.inf
+    z[2, rng.choice(V, 300, replace=False)] = 1.25
+    tdt = torch.bfloat16 if dtype == synth.BF16 else torch.float32
+    zt = torch.tensor(z, device="cuda").to(tdt)
+    zh = raw(zt, torch)
+    ctx = adasd.Context(B, V, 1, dtype=dtype, list_capacity=8)
+    ws = (float(np.float32(0.9)), 50, float(np.float32(0.9)))
+    ctx.set_warpers(*ws)
+    u = torch.tensor([0.2, 0.4, 0.6, 0.8], device="cuda")
+    H = torch.zeros(B, device="cuda")
+    lse = torch.zeros(B, device="cuda")
+    tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.draft_entropy(zt, H, u=u, token_out=tok, lse_out=lse)
+    torch.cuda.synchronize()
+    assert torch.isnan(H[0]) and int(tok[0]) == -1
+    for b in range(1, B):
+        zw, _, band = oracle.warp(zh[b], *ws, band=5e-7)
+        assert band < 1e-6
+        o = oracle.draft_step(zw, float(u[b]), 0.0)
+        assert abs(float(H[b]) - o["H"]) < TOL and abs(float(lse[b]) - o["lse"]) < TOL, (b, float(H[b]), o)
+        assert int(tok[b]) == o["token"] or o["margin"] < 2e-6, (b, int(tok[b]), o)
+    kept1 = np.isfinite(oracle.warp(zh[1], *ws)[0]).sum()
+    assert kept1 <= 10 and np.isfinite(oracle.warp(zh[2], *ws)[0]).sum() == 300      # ties stay together
+    assert ctx.status() == adasd.STATUS_NAN
