@@ -8,14 +8,16 @@
  * acceptance probability P(A|d_i) and the first-rejection accept scan (Sec. 4.4,
  * Algorithm 1), the update of the three lists L_E^R, L_D^A, L_D^R and of the
  * generation threshold T_G (Algorithm 1, step 3), and vanilla speculative sampling
- * (Sec. 2.1.3) as the comparison mode.
+ * (Sec. 2.1.3) as the comparison mode; also greedy decoding (Sec. 2.1.3), the ablation
+ * variants of Sec. 5, and the adjusted distribution of Sec. 2.1.1 (temperature, top-k,
+ * top-p) ahead of all of it.
  *
  * Conventions
  *   - Every pointer named *_dev is a DEVICE pointer owned by the caller; the library
  *     neither frees nor keeps it beyond the call.  Pointers without the suffix are
  *     host pointers.  `stream` is a cudaStream_t passed as void* (NULL = default).
- *   - Hot calls (draft_entropy, verify, update_thresholds, vanilla_verify,
- *     get_thresholds, reset) only enqueue kernels on `stream`: they never allocate,
+ *   - Hot calls (draft_entropy, verify, update_thresholds, vanilla_verify, greedy_verify,
+ *     gen_only_update, get_thresholds, reset) only enqueue kernels on `stream`: they never allocate,
  *     free or synchronise.  create/destroy/state_export/state_import/status do.
  *   - Logits are row-major with contiguous vocabulary; strides are in ELEMENTS.
  *     bf16 or fp32 as fixed at create time.  Rows whose base address and stride are
