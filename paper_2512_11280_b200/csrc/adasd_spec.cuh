@@ -31,7 +31,8 @@
 //    T_G; vanilla: longest accepted prefix) of completed sequences, off everybody's critical
 //    path; AdaSD tails are handed to the idle tail warps of the cluster's other CTAs.
 //
-// The CTA has 16 warps of 128 registers per thread: the whole register file.
+// The CTA has 16 warps of 128 registers per thread: the whole register file (136 per compute
+// thread and 104 per service thread after setmaxnreg).
 //
 // Tensor memory: 512 columns x 128 lanes of 32 bits, allocated once per CTA by the control warp.
 // A warp may only touch the 32 lanes of its quarter (warp index mod 4), so the three compute
@@ -526,12 +527,15 @@ spec_verify_kernel(VerifyParams p, ClusterGeom gq) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem0 = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_base);
 
-    // 512 threads x 128 registers fill the register file: every warp keeps what it started with
-    // (the compute warps' kept 2^t values take at most 80 registers now that the head of a position
-    // waits in tensor memory; the tail warp's float64 finalisation needs about as many).
-
-    if (warp < kSW) asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
-    else asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+    // 512 threads x 128 registers fill the register file.  The service warpgroup hands 24 registers a
+    // thread to the three compute warpgroups (8 each): setmaxnreg draws on what the CTA was launched
+    // with, so what one side gains the other must have given up first.  With the head of a position
+    // in tensor memory the compute warps keep at most 80 registers of 2^t values, and 136 leave
+    // them without spills; the tail warp's float64 finalisation and the queue workers' KDE loop get
+    // by on 104 (measured on one GPU: 144 / 80, 136 / 104, 128 / 128 and 152 / 56 give 0.4933,
+    // 0.4898, 0.4937 and 0.4955 ms on the largest workload).
+    if (warp < kSW) asm volatile("setmaxnreg.inc.sync.aligned.u32 136;");
+    else asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     bool alive = true;         // false after a wait expired: this warp stops waiting and copying
     auto expired = [&]() {
         alive = false;
